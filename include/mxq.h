@@ -1,0 +1,169 @@
+/*
+ * mxq.h -- C ABI of libmxq: block-wise microscaling (MX) quantization, Slice-and-Scale
+ * conversion, reconstruction and fused fake-quant for MF-QAT, as CUDA kernels for sm_100a.
+ *
+ * Method (section / equation numbers of the MF-QAT paper, equations counted in order of
+ * appearance):
+ *   Eq. 1  (Sec. 3.3)  shared_exp = floor(log2 max_i |V_i|) - e_max(f),  X = 2^shared_exp
+ *   Eq. 2-3 (Sec. 3.3) P_i = quantize_f(V_i / X);  MXINT: P_i = clip_b(Round(V_i / X))
+ *   Eq. 4  (Sec. 3.3)  SSMXINT: P_l = clip(Round(P_h / 2^de)),  X_l = X_h 2^de,  de = b_h - b_l
+ *   Eq. 5  (Sec. 3.4)  SSMXFP:  P_l = quantize_{eta_l,mu_l}(P_h / 2^de),  X_l = X_h 2^de,
+ *                      de = e_max(eta_h) - e_max(eta_l)
+ *   Eq. 6  (Sec. 3.5)  W_A = Q_A(W_fp),  W_t = Q_{A->t}(W_A), straight-through gradients
+ *   reconstruction (Sec. 3.3, Notation)  V^_i = X P_i
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller.  Tensor and code buffers
+ *     (src, dst, codes, out_codes, grad_*) must be 32-byte aligned (the kernels use 256-bit
+ *     global accesses); scale buffers must be 16-byte aligned.  The library enqueues work on
+ *     `stream` and returns without synchronising.  Unless an entry point says otherwise it
+ *     allocates nothing.
+ *   - `n` is the number of elements; it must be a multiple of `block`.  Blocks are runs
+ *     of `block` consecutive elements of the flat array (for a row-major matrix whose inner
+ *     dimension is a multiple of `block`: along the row).  n == 0 returns MXQ_OK at once.
+ *   - The return value is an mxq_status.  Errors detectable on the host (bad enum, null
+ *     or misaligned pointer, bad size) are reported before anything is launched;
+ *     MXQ_ERR_CUDA reports a failed launch (cudaGetLastError()).
+ *   - Scales: uint8 scales[n / block], E8M0: byte = shared_exp + 127 with shared_exp
+ *     clamped to [-127, 127]; an all-zero block stores 0; a block that holds a NaN or an
+ *     infinity stores 0xFF with all-zero codes, stays 0xFF through mxq_slice_scale and
+ *     reconstructs to quiet NaNs.
+ *   - Codes: per block, the codes form a little-endian bitstream: element i of the tensor
+ *     occupies bits [i*bits, (i+1)*bits) of the code buffer (4-bit: element 2j in the low
+ *     nibble of byte j; 6-bit: 4 codes per 3 bytes; 8-bit: one byte each).  MXINT codes are
+ *     two's-complement `bits`-bit integers in [-(2^(bits-1)-1), 2^(bits-1)-1]; MXFP codes
+ *     are sign | exponent | mantissa with the sign in the top bit.  FP8 E4M3 follows the OCP
+ *     encoding (S.1111.111 = NaN, never produced); the other MXFP element formats have no
+ *     special codes.
+ *   - e_max(MXINT b) = b - 2, e_max(MXFP eta) = 2^(eta-1).  MXINT rounding is to nearest
+ *     with ties away from zero and a symmetric clip; MXFP rounding is to nearest even
+ *     with saturation to the largest finite magnitude, subnormals kept, sign of zero kept.
+ */
+#ifndef MXQ_H
+#define MXQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque here so that the header needs no CUDA include: pass a cudaStream_t. */
+typedef void *mxq_stream;
+
+typedef enum { MXQ_F32 = 0, MXQ_BF16 = 1 } mxq_dtype;
+
+typedef enum {
+    MXQ_INT8 = 0, MXQ_INT6 = 1, MXQ_INT4 = 2,
+    MXQ_FP8_E4M3 = 3, MXQ_FP6_E3M2 = 4, MXQ_FP6_E2M3 = 5, MXQ_FP4_E2M1 = 6,
+    MXQ_INT7 = 7, MXQ_INT5 = 8, MXQ_INT3 = 9, MXQ_INT2 = 10,
+    MXQ_FP7_E3M3 = 11, MXQ_FP5_E2M2 = 12,
+    MXQ_FORMAT_COUNT = 13
+} mxq_format;
+
+typedef enum { MXQ_FQ_DIRECT = 0, MXQ_FQ_VIA_ANCHOR = 1 } mxq_fq_mode;
+
+typedef enum {
+    MXQ_OK = 0,
+    MXQ_ERR_NULL = -1,    /* a required pointer is null */
+    MXQ_ERR_FORMAT = -2,  /* unknown format / dtype / mode enum */
+    MXQ_ERR_BLOCK = -3,   /* unsupported block size */
+    MXQ_ERR_SIZE = -4,    /* n is not a multiple of block, or a count is out of range */
+    MXQ_ERR_ALIGN = -5,   /* a pointer is not aligned as required (32 bytes data, 16 bytes scales) */
+    MXQ_ERR_PAIR = -6,    /* (src_fmt, dst_fmt) is not a same-family high-to-low pair */
+    MXQ_ERR_CUDA = -7,    /* a CUDA call or launch failed */
+    MXQ_ERR_TIMEOUT = -8  /* reserved: a bounded device-side wait gave up */
+} mxq_status;
+
+/* Human-readable name of a status code (static storage, never null). */
+const char *mxq_status_string(int status);
+
+/* Bits per element code of `fmt`, or 0 for an unknown format. */
+int mxq_format_bits(int fmt);
+
+/* Bytes of the packed code buffer for n elements (n * bits / 8), 0 for an unknown format. */
+size_t mxq_codes_bytes(size_t n, int fmt);
+
+/* Bytes of the scale buffer (n / block), 0 if block <= 0. */
+size_t mxq_scales_bytes(size_t n, int block);
+
+/* 1 if `block` is a supported scaling block size, else 0. */
+int mxq_block_supported(int block);
+
+/*
+ * Q_f, Eq. 1-3: quantize `n` FP32 or BF16 elements at `src` into packed codes of element
+ * format `fmt` plus one E8M0 scale per block.  Serves the 8-bit anchors (MXINT8, MXFP8
+ * E4M3) and direct quantization to any lower format.
+ *   src    [in]  device, n elements of `src_dtype`
+ *   codes  [out] device, mxq_codes_bytes(n, fmt) bytes
+ *   scales [out] device, n / block bytes
+ */
+int mxq_quantize(const void *src, int src_dtype, size_t n, int fmt, int block,
+                 void *codes, uint8_t *scales, mxq_stream stream);
+
+/*
+ * Q_{h->l}, Eq. 4 (SSMXINT) and Eq. 5 (SSMXFP): convert packed codes + scales of `src_fmt`
+ * into `dst_fmt` without reconstructing the full-precision tensor.  Both formats must
+ * belong to the same family (MXINT or MXFP) with de = e_max(src) - e_max(dst) >= 0 and
+ * bits(dst) <= bits(src); src_fmt == dst_fmt copies.  The output scale byte is
+ * min(byte + de, 254), or 0xFF for a 0xFF input.
+ *   codes, scales         [in]  device, layout as produced by mxq_quantize
+ *   out_codes, out_scales [out] device, mxq_codes_bytes(n, dst_fmt) and n / block bytes;
+ *                               must not overlap the inputs
+ */
+int mxq_slice_scale(const void *codes, const uint8_t *scales, size_t n, int block,
+                    int src_fmt, int dst_fmt, void *out_codes, uint8_t *out_scales,
+                    mxq_stream stream);
+
+/*
+ * Reconstruction V^_i = X P_i (Sec. 3.3, Notation) into FP32 or BF16, one
+ * round-to-nearest-even rounding into the output type (exact unless the result falls
+ * below the type's normal range; beyond its range it becomes +-Inf).  MXINT zero
+ * reconstructs to +0; an MXFP zero keeps its sign.
+ *   dst [out] device, n elements of `dst_dtype`
+ */
+int mxq_dequantize(const void *codes, const uint8_t *scales, size_t n, int fmt, int block,
+                   void *dst, int dst_dtype, mxq_stream stream);
+
+/*
+ * Fused fake-quant forward, Eq. 6 in reconstructed form; nothing but the result leaves
+ * the SM.  mode MXQ_FQ_DIRECT: dst = dequantize(Q_fmt(src)).  mode MXQ_FQ_VIA_ANCHOR:
+ * dst = dequantize(Q_{A->fmt}(Q_A(src))) with A = MXINT8 for MXINT targets and MXFP8 E4M3
+ * for MXFP targets.  dst has the type of src; dst == src (in place) is allowed, any other
+ * overlap is not.
+ */
+int mxq_fake_quant(const void *src, int dtype, size_t n, int fmt, int block, int mode,
+                   void *dst, mxq_stream stream);
+
+/*
+ * Straight-through estimator backward of mxq_fake_quant (Sec. 3.5): grad_in = grad_out.
+ * grad_in == grad_out is a no-op; otherwise n elements of `dtype` are copied.
+ */
+int mxq_fake_quant_bwd(const void *grad_out, int dtype, size_t n, void *grad_in,
+                       mxq_stream stream);
+
+/*
+ * Whole-model on-the-fly conversion (Sec. 3.5, Inference): mxq_slice_scale over `count`
+ * tensors in one launch.  `items` is a HOST array; every pointer inside is a device
+ * pointer with the same requirements as in mxq_slice_scale.  The item table is copied to
+ * a device-side table owned by the library (grown with cudaMalloc on first use or when
+ * `count` exceeds its capacity, reused afterwards); the host array may be freed as soon
+ * as the call returns.  Calls that share the table are ordered by `stream`; concurrent
+ * calls on different streams are not supported.
+ */
+typedef struct {
+    const void *codes;
+    const uint8_t *scales;
+    size_t n;
+    void *out_codes;
+    uint8_t *out_scales;
+} mxq_ss_item;
+
+int mxq_slice_scale_batched(const mxq_ss_item *items, int count, int block,
+                            int src_fmt, int dst_fmt, mxq_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXQ_H */

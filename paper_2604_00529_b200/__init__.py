@@ -1,0 +1,12 @@
+"""B200-native block-wise microscaling (MX) quantization for MF-QAT.
+
+The compute lives in ``libmxq.so`` (hand-written CUDA for sm_100a behind the C ABI declared in
+``include/mxq.h``).  This package is a thin ctypes binding with the same entry-point names; it
+marshals arguments and nothing else.  There is no CPU fallback: every call fails loudly when
+the library is missing or the tensors are not CUDA tensors.
+"""
+from .binding import (  # noqa: F401
+    BF16, F32, FORMATS, FQ_DIRECT, FQ_VIA_ANCHOR, MxqError, codes_bytes, dequantize, fake_quant,
+    fake_quant_bwd, format_bits, library_path, load_library, quantize, scales_bytes, slice_scale,
+    slice_scale_batched, status_string,
+)

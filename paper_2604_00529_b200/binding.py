@@ -1,0 +1,190 @@
+"""ctypes binding of libmxq.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams: tensors are passed as raw device pointers and
+the current CUDA stream's handle.  Code and scale buffers are ``torch.uint8`` tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmxq.so")
+
+F32, BF16 = 0, 1
+FQ_DIRECT, FQ_VIA_ANCHOR = 0, 1
+
+#: format name -> mxq_format enum value (include/mxq.h)
+FORMATS = {
+    "int8": 0, "int6": 1, "int4": 2, "e4m3": 3, "e3m2": 4, "e2m3": 5, "e2m1": 6,
+    "int7": 7, "int5": 8, "int3": 9, "int2": 10, "e3m3": 11, "e2m2": 12,
+}
+
+
+class MxqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (what, status_string(status)))
+
+
+class _Item(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("n", ctypes.c_size_t),
+                ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libmxq.so (built in-tree by ``python -m paper_2604_00529_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("libmxq.so is not built: run `python -m paper_2604_00529_b200.build` "
+                          "(there is no fallback path)")
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, sz, i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    L.mxq_status_string.argtypes = [i]
+    L.mxq_status_string.restype = ctypes.c_char_p
+    L.mxq_format_bits.argtypes = [i]
+    L.mxq_format_bits.restype = i
+    L.mxq_codes_bytes.argtypes = [sz, i]
+    L.mxq_codes_bytes.restype = sz
+    L.mxq_scales_bytes.argtypes = [sz, i]
+    L.mxq_scales_bytes.restype = sz
+    L.mxq_block_supported.argtypes = [i]
+    L.mxq_block_supported.restype = i
+    L.mxq_quantize.argtypes = [vp, i, sz, i, i, vp, vp, vp]
+    L.mxq_slice_scale.argtypes = [vp, vp, sz, i, i, i, vp, vp, vp]
+    L.mxq_dequantize.argtypes = [vp, vp, sz, i, i, vp, i, vp]
+    L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
+    L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
+    L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
+    for name in ("mxq_quantize", "mxq_slice_scale", "mxq_dequantize", "mxq_fake_quant", "mxq_fake_quant_bwd",
+                 "mxq_slice_scale_batched"):
+        getattr(L, name).restype = i
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return load_library().mxq_status_string(int(status)).decode()
+
+
+def format_bits(fmt: str) -> int:
+    return load_library().mxq_format_bits(FORMATS[fmt])
+
+
+def codes_bytes(n: int, fmt: str) -> int:
+    return load_library().mxq_codes_bytes(n, FORMATS[fmt])
+
+
+def scales_bytes(n: int, block: int = 32) -> int:
+    return load_library().mxq_scales_bytes(n, block)
+
+
+def _dtype_id(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("mxq tensors are float32 or bfloat16, got %s" % t.dtype)
+
+
+def _dev(t: torch.Tensor, what: str) -> int:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (libmxq has no CPU path)" % what)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % what)
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise MxqError(rc, what)
+
+
+def quantize(src: torch.Tensor, fmt: str, block: int = 32, codes: Optional[torch.Tensor] = None,
+             scales: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """mxq_quantize: returns (packed codes uint8[n*bits/8], scales uint8[n/block])."""
+    L = load_library()
+    n = src.numel()
+    if codes is None:
+        codes = torch.empty(codes_bytes(n, fmt), dtype=torch.uint8, device=src.device)
+    if scales is None:
+        scales = torch.empty(n // block if block > 0 else 0, dtype=torch.uint8, device=src.device)
+    _check(L.mxq_quantize(_dev(src, "src"), _dtype_id(src), n, FORMATS[fmt], block, _dev(codes, "codes"),
+                          _dev(scales, "scales"), _stream(stream)), "mxq_quantize")
+    return codes, scales
+
+
+def slice_scale(codes: torch.Tensor, scales: torch.Tensor, n: int, src_fmt: str, dst_fmt: str, block: int = 32,
+                out_codes: Optional[torch.Tensor] = None, out_scales: Optional[torch.Tensor] = None,
+                stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """mxq_slice_scale: anchor codes + scales -> lower-format codes + scales."""
+    L = load_library()
+    if out_codes is None:
+        out_codes = torch.empty(codes_bytes(n, dst_fmt), dtype=torch.uint8, device=codes.device)
+    if out_scales is None:
+        out_scales = torch.empty(n // block if block > 0 else 0, dtype=torch.uint8, device=codes.device)
+    _check(L.mxq_slice_scale(_dev(codes, "codes"), _dev(scales, "scales"), n, block, FORMATS[src_fmt],
+                             FORMATS[dst_fmt], _dev(out_codes, "out_codes"), _dev(out_scales, "out_scales"),
+                             _stream(stream)), "mxq_slice_scale")
+    return out_codes, out_scales
+
+
+def dequantize(codes: torch.Tensor, scales: torch.Tensor, n: int, fmt: str, block: int = 32,
+               dtype: torch.dtype = torch.float32, dst: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """mxq_dequantize: V^ = X P as float32 or bfloat16."""
+    L = load_library()
+    if dst is None:
+        dst = torch.empty(n, dtype=dtype, device=codes.device)
+    _check(L.mxq_dequantize(_dev(codes, "codes"), _dev(scales, "scales"), n, FORMATS[fmt], block, _dev(dst, "dst"),
+                            _dtype_id(dst), _stream(stream)), "mxq_dequantize")
+    return dst
+
+
+def fake_quant(src: torch.Tensor, fmt: str, block: int = 32, mode: int = FQ_DIRECT,
+               dst: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """mxq_fake_quant: quantize-dequantize in one pass (dst may be src)."""
+    L = load_library()
+    if dst is None:
+        dst = torch.empty_like(src)
+    _check(L.mxq_fake_quant(_dev(src, "src"), _dtype_id(src), src.numel(), FORMATS[fmt], block, mode,
+                            _dev(dst, "dst"), _stream(stream)), "mxq_fake_quant")
+    return dst
+
+
+def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """mxq_fake_quant_bwd: straight-through gradient (identity)."""
+    L = load_library()
+    if grad_in is None:
+        grad_in = torch.empty_like(grad_out)
+    _check(L.mxq_fake_quant_bwd(_dev(grad_out, "grad_out"), _dtype_id(grad_out), grad_out.numel(),
+                                _dev(grad_in, "grad_in"), _stream(stream)), "mxq_fake_quant_bwd")
+    return grad_in
+
+
+def slice_scale_batched(items: Sequence[Tuple[torch.Tensor, torch.Tensor, int, torch.Tensor, torch.Tensor]],
+                        src_fmt: str, dst_fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_slice_scale_batched over (codes, scales, n, out_codes, out_scales) tuples."""
+    L = load_library()
+    arr = (_Item * len(items))()
+    for k, (c, s, n, oc, os_) in enumerate(items):
+        arr[k] = _Item(_dev(c, "codes"), _dev(s, "scales"), n, _dev(oc, "out_codes"), _dev(os_, "out_scales"))
+    _check(L.mxq_slice_scale_batched(arr, len(items), block, FORMATS[src_fmt], FORMATS[dst_fmt], _stream(stream)),
+           "mxq_slice_scale_batched")

@@ -1,0 +1,132 @@
+// Global-memory access helpers: 256-bit and 128-bit vector loads/stores (sm_100a has 32-byte
+// global accesses), lane-sized ragged pieces for the sub-byte code streams, and the bitstream
+// pack/unpack of element codes in registers.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace mxq {
+
+// ---- 32-byte accesses ---------------------------------------------------------------------
+
+__device__ __forceinline__ void ld256(uint32_t (&w)[8], const void* p)
+{
+    asm volatile("ld.global.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+}
+
+__device__ __forceinline__ void st256(void* p, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
+// ---- compile-time sized pieces --------------------------------------------------------------
+
+// Largest power of two (<= 32) dividing `bytes`: the alignment every lane's piece keeps when
+// lanes own consecutive pieces of `bytes` bytes starting from a 32-byte aligned base.
+__host__ __device__ constexpr int piece_align(int bytes)
+{
+    int a = 1;
+    while (a < 32 && bytes % (a * 2) == 0) a *= 2;
+    return a;
+}
+
+// Load NW 32-bit words (NW*4 bytes) from `p`, which is aligned to piece_align(NW*4).
+template <int NW>
+__device__ __forceinline__ void load_words(uint32_t (&w)[NW], const void* p)
+{
+    constexpr int A = piece_align(NW * 4);
+    const char* c = static_cast<const char*>(p);
+    if constexpr (A == 32) {
+#pragma unroll
+        for (int i = 0; i < NW; i += 8) {
+            uint32_t t[8];
+            ld256(t, c + i * 4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[i + j] = t[j];
+        }
+    } else if constexpr (A == 16) {
+#pragma unroll
+        for (int i = 0; i < NW; i += 4) {
+            uint4 t = *reinterpret_cast<const uint4*>(c + i * 4);
+            w[i] = t.x; w[i + 1] = t.y; w[i + 2] = t.z; w[i + 3] = t.w;
+        }
+    } else if constexpr (A == 8) {
+#pragma unroll
+        for (int i = 0; i < NW; i += 2) {
+            uint2 t = *reinterpret_cast<const uint2*>(c + i * 4);
+            w[i] = t.x; w[i + 1] = t.y;
+        }
+    } else {
+        static_assert(A == 4, "pieces are whole words");
+#pragma unroll
+        for (int i = 0; i < NW; ++i) w[i] = *reinterpret_cast<const uint32_t*>(c + i * 4);
+    }
+}
+
+// Store the low NB bytes of the word array to `p`, which is aligned to piece_align(NB).
+template <int NB, int NW>
+__device__ __forceinline__ void store_bytes(void* p, const uint32_t (&w)[NW])
+{
+    static_assert(NW * 4 >= NB, "not enough words");
+    constexpr int A = piece_align(NB);
+    char* c = static_cast<char*>(p);
+    if constexpr (A == 32) {
+#pragma unroll
+        for (int i = 0; i < NB / 4; i += 8) {
+            uint32_t t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t[j] = w[i + j];
+            st256(c + i * 4, t);
+        }
+    } else if constexpr (A == 16) {
+#pragma unroll
+        for (int i = 0; i < NB / 4; i += 4)
+            *reinterpret_cast<uint4*>(c + i * 4) = make_uint4(w[i], w[i + 1], w[i + 2], w[i + 3]);
+    } else if constexpr (A == 8) {
+#pragma unroll
+        for (int i = 0; i < NB / 4; i += 2)
+            *reinterpret_cast<uint2*>(c + i * 4) = make_uint2(w[i], w[i + 1]);
+    } else if constexpr (A == 4) {
+#pragma unroll
+        for (int i = 0; i < NB / 4; ++i) *reinterpret_cast<uint32_t*>(c + i * 4) = w[i];
+    } else if constexpr (A == 2) {
+#pragma unroll
+        for (int i = 0; i < NB / 2; ++i)
+            *reinterpret_cast<uint16_t*>(c + i * 2) = (uint16_t)(w[i / 2] >> ((i & 1) * 16));
+    } else {
+#pragma unroll
+        for (int i = 0; i < NB; ++i)
+            *reinterpret_cast<uint8_t*>(c + i) = (uint8_t)(w[i / 4] >> ((i & 3) * 8));
+    }
+}
+
+// ---- bitstream of element codes in registers -------------------------------------------------
+
+// Words needed for N codes of BITS bits.
+__host__ __device__ constexpr int code_words(int n, int bits) { return (n * bits + 31) / 32; }
+
+// Insert code number I (BITS wide, already masked) into the little-endian bitstream w[].
+template <int BITS, int I, int NW>
+__device__ __forceinline__ void put_code(uint32_t (&w)[NW], uint32_t code)
+{
+    constexpr int off = I * BITS, wi = off >> 5, sh = off & 31;
+    if constexpr (sh == 0) w[wi] = code;
+    else w[wi] |= code << sh;
+    if constexpr (sh + BITS > 32) w[wi + 1] = code >> (32 - sh);
+}
+
+// Extract code number I.
+template <int BITS, int I, int NW>
+__device__ __forceinline__ uint32_t get_code(const uint32_t (&w)[NW])
+{
+    constexpr int off = I * BITS, wi = off >> 5, sh = off & 31;
+    constexpr uint32_t mask = (1u << BITS) - 1u;
+    if constexpr (sh + BITS <= 32) return (w[wi] >> sh) & mask;
+    else return ((w[wi] >> sh) | (w[wi + 1] << (32 - sh))) & mask;
+}
+
+}  // namespace mxq

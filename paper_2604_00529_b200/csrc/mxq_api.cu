@@ -1,0 +1,233 @@
+// The C ABI of libmxq (declared in include/mxq.h): argument validation on the host, then the
+// per-operation launchers.  Nothing here synchronises the device.
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "mxq_kernels.cuh"
+#include "mxq_launch.h"
+
+namespace mxq {
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceInfo {
+    int sm_count = 0;
+};
+
+std::mutex g_mutex;
+DeviceInfo g_dev[kMaxDevices];
+
+int current_device()
+{
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) return -1;
+    return d;
+}
+
+int sm_count(int dev)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_dev[dev].sm_count == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
+        g_dev[dev].sm_count = n;
+    }
+    return g_dev[dev].sm_count;
+}
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+inline bool valid_format(int f) { return fmt_info(f).kind >= 0; }
+inline bool valid_dtype(int t) { return t == MXQ_F32 || t == MXQ_BF16; }
+inline bool valid_block(int b) { return b == 16 || b == 32 || b == 64 || b == 128; }
+
+// Checks shared by the tensor entry points; returns MXQ_OK or the first violation.
+int check_sizes(size_t n, int block)
+{
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (n % (size_t)block) return MXQ_ERR_SIZE;
+    return MXQ_OK;
+}
+
+// Device-side item table of the batched conversion: library-owned scratch, one per device.
+struct ItemTable {
+    SsDeviceItem* dev = nullptr;
+    int capacity = 0;
+};
+ItemTable g_table[kMaxDevices];
+
+}  // namespace
+
+int grid_for(const void* kernel, size_t ntiles)
+{
+    const int dev = current_device();
+    const int sms = dev >= 0 ? sm_count(dev) : 1;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0)
+        per_sm = 1;
+    const size_t wave = (size_t)sms * (size_t)per_sm;
+    const size_t need = (ntiles + kWarpsPerCta - 1) / kWarpsPerCta;
+    const size_t g = need < wave ? need : wave;
+    return (int)(g ? g : 1);
+}
+
+}  // namespace mxq
+
+using namespace mxq;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+const char* mxq_status_string(int status)
+{
+    switch (status) {
+    case MXQ_OK: return "MXQ_OK";
+    case MXQ_ERR_NULL: return "MXQ_ERR_NULL: a required pointer is null";
+    case MXQ_ERR_FORMAT: return "MXQ_ERR_FORMAT: unknown format, dtype or mode";
+    case MXQ_ERR_BLOCK: return "MXQ_ERR_BLOCK: unsupported block size";
+    case MXQ_ERR_SIZE: return "MXQ_ERR_SIZE: element count is not a multiple of the block size, or a count is out of range";
+    case MXQ_ERR_ALIGN: return "MXQ_ERR_ALIGN: a pointer is not aligned (32 bytes for tensors and codes, 16 for scales)";
+    case MXQ_ERR_PAIR: return "MXQ_ERR_PAIR: not a same-family high-to-low format pair";
+    case MXQ_ERR_CUDA: return "MXQ_ERR_CUDA: a CUDA call or kernel launch failed";
+    case MXQ_ERR_TIMEOUT: return "MXQ_ERR_TIMEOUT: a bounded device-side wait gave up";
+    default: return "unknown mxq status";
+    }
+}
+
+int mxq_format_bits(int fmt) { return valid_format(fmt) ? fmt_info(fmt).bits : 0; }
+
+size_t mxq_codes_bytes(size_t n, int fmt) { return valid_format(fmt) ? n * (size_t)fmt_info(fmt).bits / 8 : 0; }
+
+size_t mxq_scales_bytes(size_t n, int block) { return block > 0 ? n / (size_t)block : 0; }
+
+int mxq_block_supported(int block) { return valid_block(block) ? 1 : 0; }
+
+int mxq_quantize(const void* src, int src_dtype, size_t n, int fmt, int block, void* codes, uint8_t* scales,
+                 mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(src_dtype)) return MXQ_ERR_FORMAT;
+    if (int rc = check_sizes(n, block)) return rc;
+    if (n == 0) return MXQ_OK;
+    if (!src || !codes || !scales) return MXQ_ERR_NULL;
+    if (!aligned(src, 32) || !aligned(codes, 32) || !aligned(scales, 16)) return MXQ_ERR_ALIGN;
+    return launch_quantize(src, src_dtype, n, fmt, block, codes, scales, static_cast<cudaStream_t>(stream));
+}
+
+int mxq_slice_scale(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt,
+                    void* out_codes, uint8_t* out_scales, mxq_stream stream)
+{
+    if (!valid_format(src_fmt) || !valid_format(dst_fmt)) return MXQ_ERR_FORMAT;
+    if (int rc = check_sizes(n, block)) return rc;
+    if (n % 32) return MXQ_ERR_SIZE;
+    if (!ss_pair_ok(src_fmt, dst_fmt)) return MXQ_ERR_PAIR;
+    if (n == 0) return MXQ_OK;
+    if (!codes || !scales || !out_codes || !out_scales) return MXQ_ERR_NULL;
+    if (!aligned(codes, 32) || !aligned(out_codes, 32) || !aligned(scales, 16) || !aligned(out_scales, 16))
+        return MXQ_ERR_ALIGN;
+    return launch_slice_scale(codes, scales, n, block, src_fmt, dst_fmt, out_codes, out_scales,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int mxq_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dst_dtype,
+                   mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(dst_dtype)) return MXQ_ERR_FORMAT;
+    if (int rc = check_sizes(n, block)) return rc;
+    if (n % 32) return MXQ_ERR_SIZE;
+    if (n == 0) return MXQ_OK;
+    if (!codes || !scales || !dst) return MXQ_ERR_NULL;
+    if (!aligned(codes, 32) || !aligned(dst, 32) || !aligned(scales, 16)) return MXQ_ERR_ALIGN;
+    return launch_dequantize(codes, scales, n, fmt, block, dst, dst_dtype, static_cast<cudaStream_t>(stream));
+}
+
+int mxq_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, int mode, void* dst, mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(dtype)) return MXQ_ERR_FORMAT;
+    if (mode != MXQ_FQ_DIRECT && mode != MXQ_FQ_VIA_ANCHOR) return MXQ_ERR_FORMAT;
+    if (int rc = check_sizes(n, block)) return rc;
+    if (n == 0) return MXQ_OK;
+    if (!src || !dst) return MXQ_ERR_NULL;
+    if (!aligned(src, 32) || !aligned(dst, 32)) return MXQ_ERR_ALIGN;
+    return launch_fake_quant(src, dtype, n, fmt, block, mode, dst, static_cast<cudaStream_t>(stream));
+}
+
+int mxq_fake_quant_bwd(const void* grad_out, int dtype, size_t n, void* grad_in, mxq_stream stream)
+{
+    if (!valid_dtype(dtype)) return MXQ_ERR_FORMAT;
+    if (n == 0) return MXQ_OK;
+    if (!grad_out || !grad_in) return MXQ_ERR_NULL;
+    if (!aligned(grad_out, 32) || !aligned(grad_in, 32)) return MXQ_ERR_ALIGN;
+    if (grad_out == grad_in) return MXQ_OK;
+    return launch_copy(grad_out, n * (dtype == MXQ_F32 ? 4u : 2u), grad_in, static_cast<cudaStream_t>(stream));
+}
+
+int mxq_slice_scale_batched(const mxq_ss_item* items, int count, int block, int src_fmt, int dst_fmt,
+                            mxq_stream stream)
+{
+    if (!valid_format(src_fmt) || !valid_format(dst_fmt)) return MXQ_ERR_FORMAT;
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (block < 32) return MXQ_ERR_BLOCK;          // the batched sweep keeps one scale per code unit or fewer
+    if (!ss_pair_ok(src_fmt, dst_fmt)) return MXQ_ERR_PAIR;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+
+    std::vector<SsDeviceItem> host;
+    host.reserve((size_t)count);
+    size_t tiles = 0;
+    for (int i = 0; i < count; ++i) {
+        const mxq_ss_item& it = items[i];
+        if (it.n % (size_t)block || it.n % 32) return MXQ_ERR_SIZE;
+        if (it.n == 0) continue;
+        if (!it.codes || !it.scales || !it.out_codes || !it.out_scales) return MXQ_ERR_NULL;
+        if (!aligned(it.codes, 32) || !aligned(it.out_codes, 32) || !aligned(it.scales, 16) ||
+            !aligned(it.out_scales, 16))
+            return MXQ_ERR_ALIGN;
+        SsDeviceItem d;
+        d.codes = static_cast<const uint8_t*>(it.codes);
+        d.scales = it.scales;
+        d.out_codes = static_cast<uint8_t*>(it.out_codes);
+        d.out_scales = it.out_scales;
+        d.nunits = it.n / 32;
+        d.nscales = it.n / (size_t)block;
+        d.tile_begin = tiles;
+        tiles += ss_batched_tiles(d.nunits);
+        host.push_back(d);
+    }
+    if (host.empty()) return MXQ_OK;
+
+    const int dev = current_device();
+    if (dev < 0) return MXQ_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SsDeviceItem* table = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ItemTable& t = g_table[dev];
+        if (t.capacity < (int)host.size()) {
+            // grow: the old table may still be read by an earlier launch on this stream, so free it
+            // only after that work has drained
+            if (t.dev) {
+                if (cudaStreamSynchronize(s) != cudaSuccess) return MXQ_ERR_CUDA;
+                cudaFree(t.dev);
+                t.dev = nullptr;
+                t.capacity = 0;
+            }
+            int cap = 256;
+            while (cap < (int)host.size()) cap *= 2;
+            if (cudaMalloc(&t.dev, sizeof(SsDeviceItem) * (size_t)cap) != cudaSuccess) return MXQ_ERR_CUDA;
+            t.capacity = cap;
+        }
+        table = t.dev;
+    }
+    // pageable source: the runtime stages the bytes before returning, so `host` may go out of scope
+    if (cudaMemcpyAsync(table, host.data(), sizeof(SsDeviceItem) * host.size(), cudaMemcpyHostToDevice, s) !=
+        cudaSuccess)
+        return MXQ_ERR_CUDA;
+    return launch_slice_scale_batched(table, (int)host.size(), tiles, src_fmt, dst_fmt, s);
+}
+
+}  // extern "C"
+#pragma GCC visibility pop

@@ -1,0 +1,37 @@
+// Launcher of the reconstruction V^ = X P (Sec. 3.3, Notation).
+#include "mxq_kernels.cuh"
+#include "mxq_launch.h"
+
+namespace mxq {
+namespace {
+
+constexpr int kU = 1;
+
+template <class F, class T>
+int run(const void* codes, const uint8_t* scales, size_t n, int block, void* dst, cudaStream_t stream)
+{
+    auto kern = dequantize_kernel<F, T, kU>;
+    const size_t nunits = n / 32;
+    const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
+    int shift = 0, per_unit = 1;
+    if (block == 16) per_unit = 2;
+    else while ((32 << shift) < block) ++shift;
+    kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(static_cast<const uint8_t*>(codes), scales,
+                                                                        nunits, shift, per_unit,
+                                                                        static_cast<uint8_t*>(dst));
+    return MXQ_CHECK_LAUNCH();
+}
+
+}  // namespace
+
+int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
+                      cudaStream_t stream)
+{
+    MXQ_DISPATCH_FORMAT(fmt, {
+        if (dtype == MXQ_F32) return run<F, F32>(codes, scales, n, block, dst, stream);
+        return run<F, BF16>(codes, scales, n, block, dst, stream);
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+}  // namespace mxq

@@ -1,0 +1,650 @@
+// The streaming kernels of libmxq.  Common shape: every lane owns a "unit" of 32 bytes of the
+// widest stream it touches (one 256-bit global access), a warp sweeps tiles of 32*U consecutive
+// units, and warps stride over the tiles of the tensor (persistent grid sized from the SM count).
+//
+//   quantize / fake_quant : unit = 32 B of FP32/BF16 input (8 / 16 elements); a block of 32
+//                           elements spans 4 / 2 adjacent lanes, whose maxima meet by xor-shuffles.
+//   slice_scale           : unit = 32 element codes = one block per lane, no cross-lane traffic.
+//   dequantize            : unit = 32 element codes in, 64 / 128 B out.
+//
+// All of them are bound by HBM traffic; the instruction budget per element is what the code
+// below is shaped around (packed 16-bit maxima, round-down FFMA instead of float->int
+// conversions, SWAR on four 8-bit codes per register, the sm_100a narrowing cvt instructions).
+#pragma once
+#include <cstdint>
+#include <utility>
+#include <cuda_runtime.h>
+
+#include "mxq_access.cuh"
+#include "mxq_codec.cuh"
+
+namespace mxq {
+
+constexpr int kThreads = 256;
+constexpr int kWarpsPerCta = kThreads / 32;
+
+template <int N, class Fn>
+__device__ __forceinline__ void static_for(Fn&& fn)
+{
+    [&]<int... I>(std::integer_sequence<int, I...>) { (fn(std::integral_constant<int, I>{}), ...); }
+    (std::make_integer_sequence<int, N>{});
+}
+
+// ------------------------------------------------------------------------------------------
+// Source element types
+// ------------------------------------------------------------------------------------------
+
+struct F32 {
+    static constexpr int id = MXQ_F32;
+    static constexpr int size = 4;
+    static constexpr int epl = 8;     // elements per 32-byte lane unit
+};
+struct BF16 {
+    static constexpr int id = MXQ_BF16;
+    static constexpr int size = 2;
+    static constexpr int epl = 16;
+};
+
+// Element i of a lane unit as FP32 (exact widening for BF16).
+template <class T, int I>
+__device__ __forceinline__ float unit_elem(const uint32_t (&w)[8])
+{
+    if constexpr (T::size == 4) return __uint_as_float(w[I]);
+    else return __uint_as_float((I & 1) ? (w[I >> 1] & 0xFFFF0000u) : (w[I >> 1] << 16));
+}
+
+__device__ __forceinline__ float max3_abs_nan(float a, float b, float c)
+{
+    float d;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(fabsf(a)), "f"(fabsf(b)), "f"(fabsf(c)));
+    return d;
+}
+
+// FP32 bit pattern of max |element| over the lane unit; any NaN yields a NaN pattern, an
+// infinity the infinity pattern (both >= 0x7F800000, both larger than every finite pattern).
+template <class T>
+__device__ __forceinline__ uint32_t unit_amax_bits(const uint32_t (&w)[8])
+{
+    if constexpr (T::size == 4) {
+        float m0 = max3_abs_nan(__uint_as_float(w[0]), __uint_as_float(w[1]), __uint_as_float(w[2]));
+        float m1 = max3_abs_nan(__uint_as_float(w[3]), __uint_as_float(w[4]), __uint_as_float(w[5]));
+        float m2 = max3_abs_nan(__uint_as_float(w[6]), __uint_as_float(w[7]), m0);
+        float m;
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(m) : "f"(m1), "f"(m2));
+        return __float_as_uint(m) & 0x7FFFFFFFu;
+    } else {
+        // BF16 magnitudes are ordered like their 15-bit patterns: packed 16-bit integer maxima.
+        constexpr uint32_t kAbs = 0x7FFF7FFFu;
+        uint32_t a = __vimax3_s16x2(w[0] & kAbs, w[1] & kAbs, w[2] & kAbs);
+        uint32_t b = __vimax3_s16x2(w[3] & kAbs, w[4] & kAbs, w[5] & kAbs);
+        uint32_t c = __vimax3_s16x2(w[6] & kAbs, w[7] & kAbs, a);
+        uint32_t m = __vmaxu2(b, c);
+        return max(m << 16, m & 0xFFFF0000u);
+    }
+}
+
+template <int LPB>
+__device__ __forceinline__ uint32_t group_max(uint32_t v)
+{
+#pragma unroll
+    for (int o = 1; o < LPB; o <<= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// Q_f: quantize (Eq. 1-3)
+// ------------------------------------------------------------------------------------------
+
+// Codes of one lane unit, packed as a little-endian bitstream.
+template <class T, class F, int NW>
+__device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv, uint32_t (&out)[NW])
+{
+    static_for<T::epl / 2>([&](auto i) {
+        constexpr int I = decltype(i)::value;
+        uint2 c = quantize_pair<F>(unit_elem<T, 2 * I>(w), unit_elem<T, 2 * I + 1>(w), inv);
+        if constexpr (F::bits == 8) {
+            // two bytes at a time
+            constexpr int wi = I / 2, sh = (I & 1) * 16;
+            uint32_t pair = c.x | (c.y << 8);
+            if constexpr (sh == 0) out[wi] = pair;
+            else out[wi] |= pair << 16;
+        } else {
+            put_code<F::bits, 2 * I>(out, c.x);
+            put_code<F::bits, 2 * I + 1>(out, c.y);
+        }
+    });
+}
+
+template <class T, class F, int BLOCK, int U>
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes,
+                uint8_t* __restrict__ scales)
+{
+    constexpr int LPB = BLOCK / T::epl;                 // lanes per block
+    static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
+    constexpr int OB = T::epl * F::bits / 8;            // code bytes per lane unit
+    constexpr int NW = code_words(T::epl, F::bits);
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+
+    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+        const size_t u0 = tile * (32 * U) + lane;
+        uint32_t w[U][8];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit < nunits) ld256(w[u], src + unit * 32);
+            else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[u][j] = 0;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
+            const BlockScale s = block_scale<F>(amax);
+            uint32_t out[NW];
+            quantize_unit<T, F>(w[u], s.inv, out);
+            if (s.byte == 0xFFu) {
+#pragma unroll
+                for (int j = 0; j < NW; ++j) out[j] = 0;
+            }
+            if (unit < nunits) {
+                store_bytes<OB>(codes + unit * OB, out);
+                if (lane % LPB == 0) scales[unit / LPB] = (uint8_t)s.byte;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Fused fake-quant forward (Eq. 6 in reconstructed form)
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float fma_keep_plus_zero(float a, float b)
+{
+    // a * b + (+0): turns a -0 product into +0 and changes nothing else
+    float d;
+    asm("fma.rn.f32 %0, %1, %2, 0f00000000;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// two FP32 values out of a packed narrow-float pair produced by quantize_fp_hw_pair
+template <class F>
+__device__ __forceinline__ float2 widen_hw_pair(uint32_t d)
+{
+    uint32_t h2;
+    if constexpr (F::id == MXQ_FP8_E4M3) asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)d));
+    else if constexpr (F::id == MXQ_FP6_E3M2) asm("cvt.rn.f16x2.e3m2x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)d));
+    else if constexpr (F::id == MXQ_FP6_E2M3) asm("cvt.rn.f16x2.e2m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)d));
+    else asm("{ .reg .b8 t; cvt.u8.u32 t, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "r"(d));
+    float2 f;
+    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h; }"
+        : "=f"(f.x), "=f"(f.y) : "r"(h2));
+    return f;
+}
+
+// Element-format value (the real number P) of two inputs after quantization, as FP32.
+//   DIRECT     : P = quantize_F(v inv)                       (inv = 2^-shared_exp of F)
+//   VIA_ANCHOR : P = Q_{A->F}(quantize_A(v inv))             (inv = 2^-shared_exp of the anchor A)
+template <class F, int MODE>
+__device__ __forceinline__ float2 fake_quant_pair(float v0, float v1, float inv)
+{
+    using A = Fmt<F::kind == KIND_INT ? MXQ_INT8 : MXQ_FP8_E4M3>;
+    constexpr bool via = MODE == MXQ_FQ_VIA_ANCHOR && F::id != A::id;
+    constexpr int de = A::emax - F::emax;
+    float2 p;
+    if constexpr (F::kind == KIND_INT) {
+        auto one = [&](float v) {
+            uint32_t q;
+            if constexpr (via) {
+                q = int_magnitude<A>(v, inv);                                  // |P_h|
+                q = min((q + (1u << (de - 1))) >> de, F::max_mag);             // Eq. 4
+            } else {
+                q = int_magnitude<F>(v, inv);
+            }
+            float qf = __uint_as_float(0x4B000000u | q) - 8388608.0f;          // exact small integer
+            return __uint_as_float(__float_as_uint(qf) | (__float_as_uint(v) & 0x80000000u));
+        };
+        p.x = one(v0);
+        p.y = one(v1);
+    } else {
+        float r0 = v0 * inv, r1 = v1 * inv;
+        if constexpr (via) {
+            // anchor codes -> exact FP16 values -> divide by 2^de (exact) -> FP32
+            uint32_t a = quantize_fp_hw_pair<A>(r0, r1);
+            uint32_t h2;
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)a));
+            constexpr uint32_t kHalf = (uint32_t)(15 - de) << 10;              // 2^-de as FP16
+            asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(h2) : "r"(kHalf | (kHalf << 16)));
+            asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h; }"
+                : "=f"(r0), "=f"(r1) : "r"(h2));
+        }
+        if constexpr (F::hw_cvt) {
+            p = widen_hw_pair<F>(quantize_fp_hw_pair<F>(r0, r1));
+        } else {
+            p.x = decode<F>(quantize_fp_alu<F>(r0));
+            p.y = decode<F>(quantize_fp_alu<F>(r1));
+        }
+    }
+    return p;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <class T, class F, int BLOCK, int MODE, int U>
+__global__ void __launch_bounds__(kThreads)
+fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may equal src
+{
+    using A = Fmt<F::kind == KIND_INT ? MXQ_INT8 : MXQ_FP8_E4M3>;
+    constexpr bool via = MODE == MXQ_FQ_VIA_ANCHOR && F::id != A::id;
+    using S = std::conditional_t<via, A, F>;            // the format whose scale Eq. 1 computes
+    constexpr int de = A::emax - F::emax;
+    constexpr int LPB = BLOCK / T::epl;
+    static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+
+    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+        const size_t u0 = tile * (32 * U) + lane;
+        uint32_t w[U][8];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit < nunits) ld256(w[u], src + unit * 32);
+            else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[u][j] = 0;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
+            const BlockScale s = block_scale<S>(amax);
+            // X of the target format: the anchor's byte moved up by de, saturating (Eq. 4-5)
+            const uint32_t byte = via ? min(s.byte + (uint32_t)de, 254u) : s.byte;
+            const float X = scale_value(byte);
+            uint32_t out[8];
+            static_for<T::epl / 2>([&](auto i) {
+                constexpr int I = decltype(i)::value;
+                const float v0 = unit_elem<T, 2 * I>(w[u]), v1 = unit_elem<T, 2 * I + 1>(w[u]);
+                float2 p = fake_quant_pair<F, MODE>(v0, v1, s.inv);
+                float y0, y1;
+                if constexpr (F::kind == KIND_INT) {          // MXINT zero reconstructs to +0
+                    y0 = fma_keep_plus_zero(p.x, X);
+                    y1 = fma_keep_plus_zero(p.y, X);
+                } else {
+                    y0 = p.x * X;
+                    y1 = p.y * X;
+                }
+                if constexpr (T::size == 4) {
+                    out[2 * I] = __float_as_uint(y0);
+                    out[2 * I + 1] = __float_as_uint(y1);
+                } else {
+                    out[I] = pack_bf16x2(y0, y1);
+                }
+            });
+            if (s.byte == 0xFFu) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+            }
+            if (unit < nunits) st256(dst + unit * 32, out);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Q_{h->l}: Slice-and-Scale (Eq. 4-5).  One lane = 32 codes.
+// ------------------------------------------------------------------------------------------
+
+// Eq. 4 on four MXINT8 codes at once (one per byte): returns the four low-format codes, one per
+// byte, in the low BL bits.  Sign-magnitude SWAR; no carry ever crosses a byte.
+template <int BL>
+__device__ __forceinline__ uint32_t ss_int8_word(uint32_t x)
+{
+    constexpr int de = 8 - BL;
+    constexpr uint32_t k01 = 0x01010101u;
+    constexpr uint32_t kH = k01 * (1u << (de - 1));            // rounding increment
+    constexpr uint32_t kLow = k01 * (0xFFu >> de);
+    constexpr uint32_t kMask = k01 * ((1u << BL) - 1u);
+    uint32_t full;                                            // 0xFF in the bytes that are negative
+    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(x));  // selector bit 3: replicate the byte's sign
+    uint32_t s1 = full & k01;
+    uint32_t a = x ^ full;                                     // |p| - s1
+    uint32_t t = a + s1 + kH;                                  // |p| + 2^(de-1) <= 160
+    uint32_t q = (t >> de) & kLow;                             // <= 2^(BL-1)
+    q -= (q >> (BL - 1)) & k01;                                // clip to 2^(BL-1) - 1
+    return ((q ^ (full & kMask)) + s1) & kMask;                // two's complement in BL bits
+}
+
+// 4 bytes holding 6-bit codes -> 24-bit stream
+__device__ __forceinline__ uint32_t squeeze6(uint32_t x)
+{
+    uint32_t y = (x & 0x003F003Fu) | ((x & 0x3F003F00u) >> 2);
+    return (y & 0x00000FFFu) | ((y >> 4) & 0x00FFF000u);
+}
+
+__device__ __forceinline__ bool has_e4m3_nan(uint32_t x)
+{
+    return (((x & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u) != 0;
+}
+
+// Eq. 5 on two E4M3 codes (low 16 bits of `pair`) through the conversion instructions:
+// exact widening to FP16, exact division by 2^de, FP32, narrowing cvt (nearest even, saturating).
+template <class FL>
+__device__ __forceinline__ uint32_t ss_e4m3_pair_hw(uint32_t pair)
+{
+    constexpr int de = 8 - FL::emax;
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)pair));
+    constexpr uint32_t kHalf = (uint32_t)(15 - de) << 10;
+    asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(h2) : "r"(kHalf | (kHalf << 16)));
+    float f0, f1;
+    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h; }"
+        : "=f"(f0), "=f"(f1) : "r"(h2));
+    return quantize_fp_hw_pair<FL>(f0, f1);
+}
+
+// Convert the 32 codes of one lane.  in: 8*FH::bits/8... words of the high format's bitstream.
+template <class FH, class FL, int NWI, int NWO>
+__device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint32_t (&out)[NWO])
+{
+    if constexpr (FH::id == FL::id) {
+#pragma unroll
+        for (int j = 0; j < NWO; ++j) out[j] = in[j];
+    } else if constexpr (FH::id == MXQ_INT8 && FL::bits == 4) {
+        // even / odd codes of 8 -> low / high nibbles of 4 bytes
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t e = __byte_perm(in[2 * j], in[2 * j + 1], 0x6420);
+            uint32_t o = __byte_perm(in[2 * j], in[2 * j + 1], 0x7531);
+            out[j] = ss_int8_word<4>(e) | (ss_int8_word<4>(o) << 4);
+        }
+    } else if constexpr (FH::id == MXQ_INT8 && FL::bits == 6) {
+        uint32_t z[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) z[j] = squeeze6(ss_int8_word<6>(in[j]));
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            out[3 * g + 0] = z[4 * g + 0] | (z[4 * g + 1] << 24);
+            out[3 * g + 1] = (z[4 * g + 1] >> 8) | (z[4 * g + 2] << 16);
+            out[3 * g + 2] = (z[4 * g + 2] >> 16) | (z[4 * g + 3] << 8);
+        }
+    } else if constexpr (FH::id == MXQ_FP8_E4M3 && FL::hw_cvt) {
+        bool nan = false;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) nan |= has_e4m3_nan(in[j]);
+        if (!nan) {
+            if constexpr (FL::bits == 4) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t b0 = ss_e4m3_pair_hw<FL>(in[2 * j]);
+                    uint32_t b1 = ss_e4m3_pair_hw<FL>(in[2 * j] >> 16);
+                    uint32_t b2 = ss_e4m3_pair_hw<FL>(in[2 * j + 1]);
+                    uint32_t b3 = ss_e4m3_pair_hw<FL>(in[2 * j + 1] >> 16);
+                    out[j] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                }
+            } else {
+                uint32_t z[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    z[j] = squeeze6(ss_e4m3_pair_hw<FL>(in[j]) | (ss_e4m3_pair_hw<FL>(in[j] >> 16) << 16));
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    out[3 * g + 0] = z[4 * g + 0] | (z[4 * g + 1] << 24);
+                    out[3 * g + 1] = (z[4 * g + 1] >> 8) | (z[4 * g + 2] << 16);
+                    out[3 * g + 2] = (z[4 * g + 2] >> 16) | (z[4 * g + 3] << 8);
+                }
+            }
+        } else {
+            // an E4M3 NaN code (never produced by the quantizer): exact scalar path
+#pragma unroll
+            for (int j = 0; j < NWO; ++j) out[j] = 0;
+            static_for<32>([&](auto i) {
+                constexpr int I = decltype(i)::value;
+                put_code<FL::bits, I>(out, ss_fp_elem<FH, FL>(get_code<FH::bits, I>(in)));
+            });
+        }
+    } else {
+        // every other pair (including non-anchor sources): element by element
+        static_for<32>([&](auto i) {
+            constexpr int I = decltype(i)::value;
+            uint32_t c = get_code<FH::bits, I>(in);
+            uint32_t d;
+            if constexpr (FH::kind == KIND_INT) d = ss_int_elem<FH, FL>(c);
+            else d = ss_fp_elem<FH, FL>(c);
+            put_code<FL::bits, I>(out, d);
+        });
+    }
+}
+
+// Scale bytes are an element-wise stream of their own: byte -> min(byte + de, 254), 0xFF kept.
+__device__ __forceinline__ uint8_t ss_scale_byte(uint32_t b, int de)
+{
+    return (uint8_t)(b == 0xFFu ? 0xFFu : min(b + (uint32_t)de, 254u));
+}
+
+// One tensor's worth of work for a warp-strided sweep; shared by the single-tensor and the
+// batched kernels.  `first`/`stride` are in tiles.
+template <class FH, class FL, int U>
+__device__ __forceinline__ void slice_scale_sweep(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                  size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
+                                                  uint8_t* __restrict__ out_scales, size_t first, size_t stride)
+{
+    constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;      // bytes per lane unit
+    constexpr int NWI = IB / 4, NWO = OB / 4;
+    constexpr int de = FH::emax - FL::emax;
+    const int lane = threadIdx.x & 31;
+    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    for (size_t tile = first; tile < ntiles; tile += stride) {
+        const size_t u0 = tile * (32 * U) + lane;
+        uint32_t w[U][NWI];
+        uint32_t sb[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
+            else {
+#pragma unroll
+                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
+            }
+            sb[u] = unit < nscales ? scales[unit] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            uint32_t out[NWO];
+            slice_scale_unit<FH, FL>(w[u], out);
+            if (unit < nunits) store_bytes<OB>(out_codes + unit * OB, out);
+            if (unit < nscales) out_scales[unit] = ss_scale_byte(sb[u], de);
+        }
+    }
+    // scale entries beyond the number of code units (block < 32): leftover element-wise pass
+    if (nscales > nunits) {
+        const size_t tid = first * 32 + lane, nthreads = stride * 32;
+        for (size_t i = nunits + tid; i < nscales; i += nthreads) out_scales[i] = ss_scale_byte(scales[i], de);
+    }
+}
+
+template <class FH, class FL, int U>
+__global__ void __launch_bounds__(kThreads)
+slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
+                   size_t nscales, uint8_t* __restrict__ out_codes, uint8_t* __restrict__ out_scales)
+{
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    slice_scale_sweep<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, warp, nwarps);
+}
+
+// Device-side item of the batched conversion (one tensor), with its place in the flattened
+// tile space of the whole batch.
+struct SsDeviceItem {
+    const uint8_t* codes;
+    const uint8_t* scales;
+    uint8_t* out_codes;
+    uint8_t* out_scales;
+    size_t nunits;
+    size_t nscales;
+    size_t tile_begin;     // first global tile index of this tensor
+};
+
+// All tensors in one launch: the tiles of every tensor are laid end to end and warps stride over
+// that global tile space, so small tensors do not leave SMs idle.
+template <class FH, class FL, int U>
+__global__ void __launch_bounds__(kThreads)
+slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, size_t total_tiles)
+{
+    constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;
+    constexpr int NWI = IB / 4, NWO = OB / 4;
+    constexpr int de = FH::emax - FL::emax;
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    int it = 0;
+    for (size_t tile = warp; tile < total_tiles; tile += nwarps) {
+        // items are sorted by tile_begin and tile only grows: advance linearly
+        while (it + 1 < count && items[it + 1].tile_begin <= tile) ++it;
+        const SsDeviceItem t = items[it];
+        const size_t u0 = (tile - t.tile_begin) * (32 * U) + lane;
+        uint32_t w[U][NWI];
+        uint32_t sb[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit < t.nunits) load_words<NWI>(w[u], t.codes + unit * IB);
+            else {
+#pragma unroll
+                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
+            }
+            sb[u] = unit < t.nscales ? t.scales[unit] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            uint32_t out[NWO];
+            slice_scale_unit<FH, FL>(w[u], out);
+            if (unit < t.nunits) store_bytes<OB>(t.out_codes + unit * OB, out);
+            if (unit < t.nscales) t.out_scales[unit] = ss_scale_byte(sb[u], de);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Reconstruction V^ = X P.  One lane = 32 codes.
+// ------------------------------------------------------------------------------------------
+
+template <class F, class T, int U>
+__global__ void __launch_bounds__(kThreads)
+dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
+                  int units_per_scale_shift, int scales_per_unit, uint8_t* __restrict__ dst)
+{
+    constexpr int IB = 4 * F::bits, NWI = IB / 4;
+    constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+        const size_t u0 = tile * (32 * U) + lane;
+        uint32_t w[U][NWI];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
+            else {
+#pragma unroll
+                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t unit = u0 + u * 32;
+            if (unit >= nunits) continue;
+            // scales_per_unit is 1 (block >= 32: one scale shared by 2^shift units) or 2 (block 16)
+            uint32_t sbyte[2];
+            if (scales_per_unit == 1) {
+                sbyte[0] = sbyte[1] = scales[unit >> units_per_scale_shift];
+            } else {
+                sbyte[0] = scales[unit * 2];
+                sbyte[1] = scales[unit * 2 + 1];
+            }
+            uint8_t* o = dst + unit * OBYTES;
+            // four 32-byte stores for FP32 (8 elements each), two for BF16 (16 elements each)
+            constexpr int EPS = 32 / T::size;
+            static_for<32 / EPS>([&](auto k) {
+                constexpr int K = decltype(k)::value;
+                const uint32_t sbk = sbyte[(K * EPS) / 16];
+                uint32_t out[8];
+                if (sbk == 0xFFu) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+                } else {
+                    const float X = scale_value(sbk);
+                    static_for<EPS / 2>([&](auto i) {
+                        constexpr int I = K * EPS + 2 * decltype(i)::value;
+                        const uint32_t c0 = get_code<F::bits, I>(w[u]), c1 = get_code<F::bits, I + 1>(w[u]);
+                        float y0 = decode<F>(c0) * X;
+                        float y1 = decode<F>(c1) * X;
+                        // an E4M3 NaN code reconstructs to the canonical quiet NaN
+                        bool n0 = false, n1 = false;
+                        if constexpr (F::has_nan) {
+                            n0 = (c0 & 0x7Fu) == 0x7Fu;
+                            n1 = (c1 & 0x7Fu) == 0x7Fu;
+                        }
+                        if constexpr (T::size == 4) {
+                            out[I - K * EPS] = n0 ? 0x7FC00000u : __float_as_uint(y0);
+                            out[I - K * EPS + 1] = n1 ? 0x7FC00000u : __float_as_uint(y1);
+                        } else {
+                            uint32_t p = pack_bf16x2(y0, y1);
+                            if (n0) p = (p & 0xFFFF0000u) | 0x7FC0u;
+                            if (n1) p = (p & 0x0000FFFFu) | 0x7FC00000u;
+                            out[(I - K * EPS) / 2] = p;
+                        }
+                    });
+                }
+                st256(o + K * 32, out);
+            });
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Straight-through backward: a plain copy
+// ------------------------------------------------------------------------------------------
+
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict__ dst)
+{
+    const size_t nunits = nbytes / 32;
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+        const size_t u0 = tile * (32 * U) + lane;
+        uint32_t w[U][8];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (u0 + u * 32 < nunits) ld256(w[u], src + (u0 + u * 32) * 32);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (u0 + u * 32 < nunits) st256(dst + (u0 + u * 32) * 32, w[u]);
+    }
+    // ragged tail (n * size need not be a multiple of 32 bytes)
+    const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
+    for (size_t i = nunits * 32 + tid; i < nbytes; i += (size_t)gridDim.x * kThreads) dst[i] = src[i];
+}
+
+}  // namespace mxq

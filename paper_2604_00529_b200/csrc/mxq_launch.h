@@ -1,0 +1,55 @@
+// Internal interface between the C ABI (argument checks, mxq_api.cu) and the per-operation
+// translation units that instantiate and launch the kernels.  Arguments are already validated.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/mxq.h"
+
+namespace mxq {
+
+// Persistent-grid size for a kernel: enough CTAs for `ntiles` warp tiles, at most one full wave
+// (SM count x resident CTAs per SM for this kernel on the current device).
+int grid_for(const void* kernel, size_t ntiles);
+
+int launch_quantize(const void* src, int dtype, size_t n, int fmt, int block, void* codes, uint8_t* scales,
+                    cudaStream_t stream);
+int launch_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, int mode, void* dst,
+                      cudaStream_t stream);
+int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt,
+                       void* out_codes, uint8_t* out_scales, cudaStream_t stream);
+int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
+                      cudaStream_t stream);
+int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
+
+// Batched Slice-and-Scale over a device-resident item table (see mxq_kernels.cuh: SsDeviceItem).
+struct SsDeviceItem;
+int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t total_tiles, int src_fmt,
+                               int dst_fmt, cudaStream_t stream);
+// tiles one tensor of `nunits` lane units occupies in the batched kernel's tile space
+size_t ss_batched_tiles(size_t nunits);
+
+// Expands the body once per element format with NAME bound to mxq::Fmt<id>.
+#define MXQ_DISPATCH_FORMAT_AS(fmt, NAME, ...)                                      \
+    switch (fmt) {                                                                  \
+    case MXQ_INT8: { using NAME = ::mxq::Fmt<MXQ_INT8>; __VA_ARGS__; } break;           \
+    case MXQ_INT7: { using NAME = ::mxq::Fmt<MXQ_INT7>; __VA_ARGS__; } break;           \
+    case MXQ_INT6: { using NAME = ::mxq::Fmt<MXQ_INT6>; __VA_ARGS__; } break;           \
+    case MXQ_INT5: { using NAME = ::mxq::Fmt<MXQ_INT5>; __VA_ARGS__; } break;           \
+    case MXQ_INT4: { using NAME = ::mxq::Fmt<MXQ_INT4>; __VA_ARGS__; } break;           \
+    case MXQ_INT3: { using NAME = ::mxq::Fmt<MXQ_INT3>; __VA_ARGS__; } break;           \
+    case MXQ_INT2: { using NAME = ::mxq::Fmt<MXQ_INT2>; __VA_ARGS__; } break;           \
+    case MXQ_FP8_E4M3: { using NAME = ::mxq::Fmt<MXQ_FP8_E4M3>; __VA_ARGS__; } break;   \
+    case MXQ_FP7_E3M3: { using NAME = ::mxq::Fmt<MXQ_FP7_E3M3>; __VA_ARGS__; } break;   \
+    case MXQ_FP6_E3M2: { using NAME = ::mxq::Fmt<MXQ_FP6_E3M2>; __VA_ARGS__; } break;   \
+    case MXQ_FP6_E2M3: { using NAME = ::mxq::Fmt<MXQ_FP6_E2M3>; __VA_ARGS__; } break;   \
+    case MXQ_FP5_E2M2: { using NAME = ::mxq::Fmt<MXQ_FP5_E2M2>; __VA_ARGS__; } break;   \
+    case MXQ_FP4_E2M1: { using NAME = ::mxq::Fmt<MXQ_FP4_E2M1>; __VA_ARGS__; } break;   \
+    default: return MXQ_ERR_FORMAT;                                                 \
+    }
+#define MXQ_DISPATCH_FORMAT(fmt, ...) MXQ_DISPATCH_FORMAT_AS(fmt, F, __VA_ARGS__)
+
+#define MXQ_CHECK_LAUNCH() (cudaGetLastError() == cudaSuccess ? MXQ_OK : MXQ_ERR_CUDA)
+
+}  // namespace mxq

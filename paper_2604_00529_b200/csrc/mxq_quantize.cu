@@ -1,0 +1,50 @@
+// Launcher of Q_f (Eq. 1-3): instantiates quantize_kernel per source type, element format and
+// block size.
+#include "mxq_kernels.cuh"
+#include "mxq_launch.h"
+
+namespace mxq {
+namespace {
+
+constexpr int kU = 2;   // lane units in flight per thread
+
+template <class T, class F, int BLOCK>
+int run(const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t stream)
+{
+    if constexpr (BLOCK < T::epl) {
+        return MXQ_ERR_BLOCK;
+    } else {
+        auto kern = quantize_kernel<T, F, BLOCK, kU>;
+        const size_t nunits = n / T::epl;
+        const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
+        kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(
+            static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(codes), scales);
+        return MXQ_CHECK_LAUNCH();
+    }
+}
+
+template <class T, class F>
+int by_block(int block, const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t stream)
+{
+    switch (block) {
+    case 16: return run<T, F, 16>(src, n, codes, scales, stream);
+    case 32: return run<T, F, 32>(src, n, codes, scales, stream);
+    case 64: return run<T, F, 64>(src, n, codes, scales, stream);
+    case 128: return run<T, F, 128>(src, n, codes, scales, stream);
+    default: return MXQ_ERR_BLOCK;
+    }
+}
+
+}  // namespace
+
+int launch_quantize(const void* src, int dtype, size_t n, int fmt, int block, void* codes, uint8_t* scales,
+                    cudaStream_t stream)
+{
+    MXQ_DISPATCH_FORMAT(fmt, {
+        if (dtype == MXQ_F32) return by_block<F32, F>(block, src, n, codes, scales, stream);
+        return by_block<BF16, F>(block, src, n, codes, scales, stream);
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+}  // namespace mxq

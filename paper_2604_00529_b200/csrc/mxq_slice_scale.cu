@@ -1,0 +1,53 @@
+// Launchers of Slice-and-Scale (Eq. 4-5): one tensor per launch, and the batched form that
+// converts a whole set of tensors in one launch.
+#include "mxq_kernels.cuh"
+#include "mxq_launch.h"
+
+namespace mxq {
+namespace {
+
+constexpr int kU = 2;
+
+}  // namespace
+
+size_t ss_batched_tiles(size_t nunits) { return (nunits + 32 * kU - 1) / (32 * kU); }
+
+int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt,
+                       void* out_codes, uint8_t* out_scales, cudaStream_t stream)
+{
+    MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, {
+            if constexpr (ss_pair_ok(FH::id, FL::id)) {
+                auto kern = slice_scale_kernel<FH, FL, kU>;
+                const size_t nunits = n / 32, nscales = n / (size_t)block;
+                const size_t ntiles = ss_batched_tiles(nunits);
+                kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(
+                    static_cast<const uint8_t*>(codes), scales, nunits, nscales, static_cast<uint8_t*>(out_codes),
+                    out_scales);
+                return MXQ_CHECK_LAUNCH();
+            } else {
+                return MXQ_ERR_PAIR;
+            }
+        });
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t total_tiles, int src_fmt,
+                               int dst_fmt, cudaStream_t stream)
+{
+    MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, {
+            if constexpr (ss_pair_ok(FH::id, FL::id)) {
+                auto kern = slice_scale_batched_kernel<FH, FL, kU>;
+                kern<<<grid_for((const void*)kern, total_tiles), kThreads, 0, stream>>>(items_dev, count, total_tiles);
+                return MXQ_CHECK_LAUNCH();
+            } else {
+                return MXQ_ERR_PAIR;
+            }
+        });
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+}  // namespace mxq

@@ -1,0 +1,296 @@
+"""GPU parity: every entry point of libmxq, called through the C-ABI binding, against the CPU
+oracle on identical seeded inputs.  Codes, scales and reconstructed values must match bit for bit
+(integer and byte work; floating point decides nothing here that both sides do not decide in the
+same exact arithmetic, so the tolerance is zero)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2604_00529_b200 as mxq
+from oracle import mxq_oracle as orc
+from paper_2604_00529_b200 import inputs
+
+from gpu_util import (ALL_FORMATS, FP_FORMATS, INT_FORMATS, MAIN_FORMATS, bits_equal, first_diff, gpu_dequantize,
+                      gpu_fake_quant, gpu_quantize, gpu_slice_scale, ss_pairs, to_dev, to_host)
+
+pytestmark = pytest.mark.gpu
+
+
+def _mixed_f32(nblk, seed, block=32):
+    """Blocks at many magnitudes with outliers; spans several warp tiles plus a ragged tail."""
+    rng = np.random.default_rng(seed)
+    scale = 2.0 ** rng.integers(-30, 30, (nblk, 1))
+    x = rng.standard_normal((nblk, block)) * scale
+    x[rng.random((nblk, block)) < 0.02] *= 40
+    x[rng.random((nblk, block)) < 0.05] = 0
+    return x.astype(np.float32).reshape(-1)
+
+
+def _oracle_packed(x, fmt, block=32):
+    c, s = orc.quantize(x, fmt, block)
+    return orc.pack(c, orc.bits(fmt)), s
+
+
+# 64 lane units per warp tile: 2051 blocks of FP32 = 8204 units = 128 tiles + a ragged tail
+NBLK = 2051
+
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS)
+@pytest.mark.parametrize("bf16", [False, True])
+def test_quantize_random(fmt, bf16):
+    x = np.concatenate([_mixed_f32(NBLK, 1), inputs.adversarial_f32()])
+    if bf16:
+        x = inputs.to_bf16_bits(x)
+    got_c, got_s = gpu_quantize(x, fmt)
+    want_c, want_s = _oracle_packed(x, fmt)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, want_c), first_diff(got_c, want_c)
+
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS)
+def test_quantize_every_bf16_pattern(fmt):
+    """All 65536 BF16 bit patterns as block elements, under pinned block maxima at several
+    exponents (non-finite patterns poison their block, which is part of the contract)."""
+    pats = np.arange(65536, dtype=np.uint16)
+    blocks = []
+    for k in (-126, -60, -9, 0, 3, 9, 90, 127):
+        pin = inputs.to_bf16_bits(np.array([1.75 * 2.0 ** k], np.float32))[0]
+        body = np.concatenate([pats, np.zeros((-65536) % 31, np.uint16)]).reshape(-1, 31)
+        blk = np.concatenate([np.full((body.shape[0], 1), pin, np.uint16), body], axis=1)
+        blocks.append(blk.reshape(-1))
+    x = np.concatenate(blocks)
+    got_c, got_s = gpu_quantize(x, fmt)
+    want_c, want_s = _oracle_packed(x, fmt)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, want_c), first_diff(got_c, want_c)
+
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS)
+def test_quantize_f32_rounding_breakpoints(fmt):
+    """FP32 inputs one ulp either side of every rounding breakpoint of the element format, at
+    several block scales (the quantizer is a monotone step function: breakpoints suffice)."""
+    tab = orc.decode_table(fmt)
+    mags = np.unique(np.abs(tab[~np.isnan(tab)]))
+    top = orc.max_value(fmt)
+    mids = (mags[:-1] + mags[1:]) / 2
+    pts = np.concatenate([mags, mids, [top + (mags[-1] - mags[-2]) / 2, top * 1.2]]).astype(np.float32)
+    pts = np.concatenate([pts, np.nextafter(pts, np.float32(np.inf)), np.nextafter(pts, np.float32(-np.inf))])
+    pts = pts[pts < 2.0 ** (orc.emax(fmt) + 1)]                 # must stay below the pinned maximum's binade
+    pts = np.concatenate([pts, -pts])
+    pin = np.float32(1.999 * 2.0 ** orc.emax(fmt))              # floor(log2) = e_max -> shared_exp = k
+    xs = []
+    for k in (-100, -17, 0, 5, 60):
+        body = np.concatenate([pts, np.zeros((-pts.size) % 31, np.float32)]).reshape(-1, 31)
+        blk = np.concatenate([np.full((body.shape[0], 1), pin, np.float32), body], axis=1)
+        xs.append((blk * np.float32(2.0 ** k)).astype(np.float32).reshape(-1))
+    x = np.concatenate(xs)
+    got_c, got_s = gpu_quantize(x, fmt)
+    want_c, want_s = _oracle_packed(x, fmt)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, want_c), first_diff(got_c, want_c)
+
+
+@pytest.mark.parametrize("block", [16, 64, 128])
+@pytest.mark.parametrize("fmt", ["int8", "int4", "e4m3", "e2m1", "e3m2"])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_quantize_other_block_sizes(fmt, block, bf16):
+    x = _mixed_f32(777, 2, block)
+    if bf16:
+        x = inputs.to_bf16_bits(x)
+    got_c, got_s = gpu_quantize(x, fmt, block)
+    want_c, want_s = _oracle_packed(x, fmt, block)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, want_c), first_diff(got_c, want_c)
+
+
+# ---------------------------------------------------------------------------------------------
+# Slice-and-Scale
+# ---------------------------------------------------------------------------------------------
+
+def _all_codes_input(src, nblk_extra=1000, seed=3):
+    """Every code value of the source format (NaN codes and -2^(b-1) included) in every lane
+    position, then random codes; scale bytes cover 0, the saturating range and 0xFF."""
+    nb = orc.bits(src)
+    rng = np.random.default_rng(seed)
+    allc = np.arange(1 << nb, dtype=np.uint8)
+    rolled = np.concatenate([np.roll(np.resize(allc, 256), r) for r in range(32)])
+    codes = np.concatenate([rolled, rng.integers(0, 1 << nb, 32 * nblk_extra).astype(np.uint8)])
+    nblk = codes.size // 32
+    scales = rng.integers(0, 256, nblk).astype(np.uint8)
+    scales[:8] = [0, 1, 248, 250, 252, 253, 254, 255]
+    return codes, scales
+
+
+@pytest.mark.parametrize("src,dst", ss_pairs(all_pairs=True), ids=lambda v: v)
+def test_slice_scale_all_codes(src, dst):
+    codes, scales = _all_codes_input(src)
+    n = codes.size
+    got_c, got_s = gpu_slice_scale(orc.pack(codes, orc.bits(src)), scales, n, src, dst)
+    want_c, want_s = orc.slice_scale(codes, scales, src, dst)
+    want_c = orc.pack(want_c, orc.bits(dst))
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, want_c), first_diff(got_c, want_c)
+
+
+@pytest.mark.parametrize("src,dst", ss_pairs(), ids=lambda v: v)
+def test_slice_scale_of_quantized_tensor(src, dst):
+    """The paper's path: anchor = Q_A(V) on the GPU, then Q_{A->t}; both stages against the oracle."""
+    x = inputs.to_bf16_bits(_mixed_f32(NBLK, 4))
+    n = x.size
+    a_c, a_s = gpu_quantize(x, src)
+    got_c, got_s = gpu_slice_scale(a_c, a_s, n, src, dst)
+    oc, os_ = orc.quantize(x, src)
+    want_c, want_s = orc.slice_scale(oc, os_, src, dst)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, orc.pack(want_c, orc.bits(dst))), first_diff(got_c, orc.pack(want_c, orc.bits(dst)))
+
+
+@pytest.mark.parametrize("block", [16, 64, 128])
+@pytest.mark.parametrize("src,dst", [("int8", "int4"), ("e4m3", "e2m3")])
+def test_slice_scale_other_block_sizes(src, dst, block):
+    rng = np.random.default_rng(block)
+    n = 128 * 301
+    codes = rng.integers(0, 255, n).astype(np.uint8)
+    codes[codes == 0x7F] = 0x7E
+    scales = rng.integers(0, 256, n // block).astype(np.uint8)
+    got_c, got_s = gpu_slice_scale(codes, scales, n, src, dst, block)
+    want_c, want_s = orc.slice_scale(codes, scales, src, dst, block)
+    assert bits_equal(got_s, want_s), first_diff(got_s, want_s)
+    assert bits_equal(got_c, orc.pack(want_c, orc.bits(dst)))
+
+
+def test_slice_scale_batched_matches_oracle():
+    """Tensors of very different sizes (one smaller than a tile) in one launch."""
+    rng = np.random.default_rng(9)
+    sizes = [32, 32 * 7, 32 * 64, 32 * 65, 32 * 4097, 32 * 1000, 32, 32 * 333]
+    for src, dst in (("int8", "int6"), ("int8", "int4"), ("e4m3", "e2m3"), ("e4m3", "e3m2"), ("e4m3", "e2m1")):
+        items, wants = [], []
+        for n in sizes:
+            codes = rng.integers(0, 256, n).astype(np.uint8)
+            codes[(codes & 0x7F) == 0x7F] &= 0xFE
+            scales = rng.integers(0, 256, n // 32).astype(np.uint8)
+            oc = torch.full((mxq.codes_bytes(n, dst) + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            os_ = torch.full((n // 32 + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+            items.append((to_dev(codes), to_dev(scales), n, oc, os_))
+            wants.append(orc.slice_scale(codes, scales, src, dst))
+        mxq.slice_scale_batched(items, src, dst)
+        mxq.slice_scale_batched(items, src, dst)      # the item table is reused
+        torch.cuda.synchronize()
+        for (c, s, n, oc, os_), (wc, ws) in zip(items, wants):
+            nb = mxq.codes_bytes(n, dst)
+            assert bits_equal(to_host(oc[:nb]), orc.pack(wc, orc.bits(dst)))
+            assert bits_equal(to_host(os_[:n // 32]), ws)
+            assert np.all(to_host(oc[nb:]) == 0xA5) and np.all(to_host(os_[n // 32:]) == 0xA5)
+
+
+# ---------------------------------------------------------------------------------------------
+# Reconstruction
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS)
+@pytest.mark.parametrize("bf16", [False, True])
+def test_dequantize_all_codes_all_scales(fmt, bf16):
+    """Every code under every scale byte (subnormal results, overflow to infinity, 0xFF -> NaN)."""
+    nb = orc.bits(fmt)
+    allc = np.resize(np.arange(1 << nb, dtype=np.uint8), 256)
+    codes = np.tile(allc, 256 * 2)                       # 8 blocks of 32 per sweep, two sweeps per scale byte
+    n = codes.size
+    scales = np.repeat(np.arange(256, dtype=np.uint8), n // 32 // 256)
+    got = gpu_dequantize(orc.pack(codes, nb), scales, n, fmt, bf16=bf16)
+    want = orc.dequantize(codes, scales, fmt, out_dtype=orc.BF16 if bf16 else orc.F32)
+    assert bits_equal(got, want), first_diff(got, want)
+
+
+@pytest.mark.parametrize("block", [16, 64, 128])
+@pytest.mark.parametrize("fmt", ["int4", "e2m3", "e4m3"])
+def test_dequantize_other_block_sizes(fmt, block):
+    rng = np.random.default_rng(block + 1)
+    n = 128 * 257
+    codes = rng.integers(0, 1 << orc.bits(fmt), n).astype(np.uint8)
+    scales = rng.integers(100, 160, n // block).astype(np.uint8)
+    for bf16 in (False, True):
+        got = gpu_dequantize(orc.pack(codes, orc.bits(fmt)), scales, n, fmt, block, bf16=bf16)
+        want = orc.dequantize(codes, scales, fmt, block, orc.BF16 if bf16 else orc.F32)
+        assert bits_equal(got, want), first_diff(got, want)
+
+
+# ---------------------------------------------------------------------------------------------
+# Fake-quant
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("fmt", ALL_FORMATS)
+@pytest.mark.parametrize("mode", [orc.FQ_DIRECT, orc.FQ_VIA_ANCHOR])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_fake_quant(fmt, mode, bf16):
+    x = np.concatenate([_mixed_f32(NBLK, 5), inputs.adversarial_f32()])
+    if bf16:
+        x = inputs.to_bf16_bits(x)
+    got = gpu_fake_quant(x, fmt, mode=mode)
+    want = orc.fake_quant(x, fmt, mode=mode)
+    assert bits_equal(got, want), first_diff(got, want)
+
+
+@pytest.mark.parametrize("fmt", ["int6", "e2m3"])
+def test_fake_quant_every_bf16_pattern(fmt):
+    pats = np.arange(65536, dtype=np.uint16)
+    blocks = []
+    for k in (-126, -9, 0, 100):
+        pin = inputs.to_bf16_bits(np.array([1.75 * 2.0 ** k], np.float32))[0]
+        body = np.concatenate([pats, np.zeros((-65536) % 31, np.uint16)]).reshape(-1, 31)
+        blocks.append(np.concatenate([np.full((body.shape[0], 1), pin, np.uint16), body], axis=1).reshape(-1))
+    x = np.concatenate(blocks)
+    for mode in (orc.FQ_DIRECT, orc.FQ_VIA_ANCHOR):
+        got = gpu_fake_quant(x, fmt, mode=mode)
+        want = orc.fake_quant(x, fmt, mode=mode)
+        assert bits_equal(got, want), first_diff(got, want)
+
+
+@pytest.mark.parametrize("block", [16, 64, 128])
+def test_fake_quant_other_block_sizes(block):
+    x = inputs.to_bf16_bits(_mixed_f32(501, 6, block))
+    for fmt in ("int4", "e2m1"):
+        for mode in (orc.FQ_DIRECT, orc.FQ_VIA_ANCHOR):
+            got = gpu_fake_quant(x, fmt, block, mode)
+            want = orc.fake_quant(x, fmt, block, mode)
+            assert bits_equal(got, want), first_diff(got, want)
+
+
+def test_fake_quant_in_place_and_backward():
+    x = inputs.to_bf16_bits(_mixed_f32(513, 7))
+    want = orc.fake_quant(x, "int4", mode=orc.FQ_VIA_ANCHOR)
+    got = gpu_fake_quant(x, "int4", mode=orc.FQ_VIA_ANCHOR, inplace=True)
+    assert bits_equal(got, want)
+    # straight-through estimator: the gradient comes back unchanged, for any length
+    for n in (1, 31, 4096, 4096 * 5 + 3):
+        g = to_dev(inputs.to_bf16_bits(np.random.default_rng(n).standard_normal(n).astype(np.float32)))
+        gi = mxq.fake_quant_bwd(g)
+        torch.cuda.synchronize()
+        assert torch.equal(gi.view(torch.int16), g.view(torch.int16))
+        assert mxq.fake_quant_bwd(g, g) is g
+    g32 = torch.randn(1000, device="cuda")
+    assert torch.equal(mxq.fake_quant_bwd(g32), g32)
+
+
+# ---------------------------------------------------------------------------------------------
+# chained entry points and degenerate sizes
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("fmt", MAIN_FORMATS)
+def test_quantize_then_dequantize_equals_fake_quant(fmt):
+    """The fused kernel and the two-kernel route agree with each other as well as with the oracle."""
+    x = inputs.to_bf16_bits(_mixed_f32(300, 8))
+    n = x.size
+    c, s = gpu_quantize(x, fmt)
+    v = gpu_dequantize(c, s, n, fmt, bf16=True)
+    assert bits_equal(v, gpu_fake_quant(x, fmt))
+
+
+def test_smallest_and_empty_inputs():
+    x = np.array([1.0] + [0.25] * 31, np.float32)
+    c, s = gpu_quantize(x, "int8")
+    wc, ws = _oracle_packed(x, "int8")
+    assert bits_equal(c, wc) and bits_equal(s, ws)
+    empty = torch.empty(0, dtype=torch.float32, device="cuda")
+    c, s = mxq.quantize(empty, "int8")
+    assert c.numel() == 0 and s.numel() == 0
+    assert mxq.fake_quant(empty, "e2m1").numel() == 0
