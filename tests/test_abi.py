@@ -1,0 +1,88 @@
+"""The C-ABI library on a machine without a GPU: it loads, exports every function the public header
+declares, and its host-side argument checks answer before anything is launched (no call here can
+reach a kernel launch: each one is rejected on the host, or has n == 0)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2604_00529_b200 as mxq
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+OK, E_NULL, E_FORMAT, E_BLOCK, E_SIZE, E_ALIGN, E_PAIR = 0, -1, -2, -3, -4, -5, -6
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "mxq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mxq_[a-z0-9_]+)\s*\(", text)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    return mxq.load_library()
+
+
+def test_every_declared_function_is_exported(L):
+    names = _declared_functions()
+    assert {"mxq_quantize", "mxq_slice_scale", "mxq_dequantize", "mxq_fake_quant", "mxq_fake_quant_bwd",
+            "mxq_slice_scale_batched"} <= set(names)
+    for name in names:
+        assert hasattr(L, name), name
+
+
+def test_size_helpers(L):
+    assert [L.mxq_format_bits(f) for f in range(13)] == [8, 6, 4, 8, 6, 6, 4, 7, 5, 3, 2, 7, 5]
+    assert L.mxq_format_bits(13) == 0 and L.mxq_format_bits(-1) == 0
+    assert L.mxq_codes_bytes(64, mxq.FORMATS["int6"]) == 48
+    assert L.mxq_codes_bytes(1 << 31, mxq.FORMATS["e2m1"]) == 1 << 30
+    assert L.mxq_scales_bytes(4096, 32) == 128 and L.mxq_scales_bytes(4096, 0) == 0
+    assert [L.mxq_block_supported(b) for b in (8, 16, 32, 48, 64, 128, 256)] == [0, 1, 1, 0, 1, 1, 0]
+    assert b"MXQ_OK" in L.mxq_status_string(0) and b"unknown" in L.mxq_status_string(-99)
+    for st in range(-8, 0):
+        assert L.mxq_status_string(st).startswith(b"MXQ_ERR_")
+
+
+def test_argument_checks_answer_on_the_host(L):
+    A = 0x1000                       # an aligned, never dereferenced address
+    q = L.mxq_quantize
+    assert q(A, 0, 64, 99, 32, A, A, None) == E_FORMAT
+    assert q(A, 7, 64, 0, 32, A, A, None) == E_FORMAT
+    assert q(A, 0, 64, 0, 48, A, A, None) == E_BLOCK
+    assert q(A, 0, 65, 0, 32, A, A, None) == E_SIZE
+    assert q(None, 0, 64, 0, 32, A, A, None) == E_NULL
+    assert q(A + 16, 0, 64, 0, 32, A, A, None) == E_ALIGN
+    assert q(A, 0, 64, 0, 32, A, A + 8, None) == E_ALIGN
+    assert q(None, 0, 0, 0, 32, None, None, None) == OK           # empty tensor: nothing to do
+    ss = L.mxq_slice_scale
+    F = mxq.FORMATS
+    assert ss(A, A, 64, 32, F["int8"], F["e2m1"], A, A, None) == E_PAIR      # families differ
+    assert ss(A, A, 64, 32, F["int4"], F["int8"], A, A, None) == E_PAIR      # low to high
+    assert ss(A, A, 64, 32, F["e2m1"], F["e2m3"], A, A, None) == E_PAIR      # codes would widen
+    assert ss(A, A, 64, 32, F["int8"], F["int4"], None, A, None) == E_NULL
+    assert ss(A, A, 64, 32, F["int8"], F["int4"], A + 4, A, None) == E_ALIGN
+    assert ss(A, A, 48, 16, F["int8"], F["int4"], A, A, None) == E_SIZE      # code units are 32 wide
+    dq = L.mxq_dequantize
+    assert dq(A, A, 64, F["int4"], 32, A, 5, None) == E_FORMAT
+    assert dq(A, None, 64, F["int4"], 32, A, 0, None) == E_NULL
+    fq = L.mxq_fake_quant
+    assert fq(A, 1, 64, F["e2m1"], 32, 2, A, None) == E_FORMAT               # unknown mode
+    assert fq(A, 1, 64, F["e2m1"], 32, 1, None, None) == E_NULL
+    bw = L.mxq_fake_quant_bwd
+    assert bw(A, 1, 64, A, None) == OK                                       # in place: no launch
+    assert bw(A, 1, 64, None, None) == E_NULL
+    for fn in (L.mxq_slice_scale_batched,):
+        assert fn(None, 3, 32, F["int8"], F["int4"], None) == E_NULL
+        assert fn(None, -1, 32, F["int8"], F["int4"], None) == E_SIZE
+        assert fn(None, 0, 32, F["int8"], F["int4"], None) == OK
+        assert fn(None, 3, 16, F["int8"], F["int4"], None) == E_BLOCK
+        assert fn(None, 3, 32, F["int8"], F["e2m1"], None) == E_PAIR
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    with pytest.raises(ValueError):
+        mxq.quantize(torch.zeros(64), "int8")
+    with pytest.raises((TypeError, ValueError)):
+        mxq.fake_quant(torch.zeros(64, dtype=torch.float16), "int8")
