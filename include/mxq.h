@@ -163,6 +163,28 @@ typedef struct {
 int mxq_slice_scale_batched(const mxq_ss_item *items, int count, int block,
                             int src_fmt, int dst_fmt, mxq_stream stream);
 
+/*
+ * The same conversion as mxq_slice_scale_batched for callers that cannot allocate device memory.
+ * (The paper has no counterpart of this entry point; it exists for the library's users.)  Some
+ * processes give all of HBM to a pool of their own at start-up, so a cudaMalloc made behind their
+ * back fails or takes memory that was promised elsewhere; others run a loop where the host must
+ * never stall, and cudaMalloc / cudaFree wait for the device.  For them the item table lives in a
+ * fixed array inside the library image: MXQ_STATIC_BATCH_MAX items, 56 KiB, present on every GPU
+ * that loads libmxq until the process exits.  This call makes no cudaMalloc, cudaFree or other
+ * allocating call, on the device or on the host heap.
+ *   - Arguments, checks and results are those of mxq_slice_scale_batched (block must be 32, 64 or
+ *     128); in addition count > MXQ_STATIC_BATCH_MAX returns MXQ_ERR_SIZE and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and keeps it; make that first call before starting any stream capture.
+ *   - All calls on one device share the one table.  Each call rewrites the entries it uses and the
+ *     kernel reads no others, so stale contents of an earlier call are harmless.  Calls ordered by
+ *     one stream are safe; two calls whose work can overlap on the GPU (different streams, no
+ *     dependency between them) race on the table and give undefined results.
+ */
+#define MXQ_STATIC_BATCH_MAX 1024
+int mxq_slice_scale_batched_static(const mxq_ss_item *items, int count, int block,
+                                   int src_fmt, int dst_fmt, mxq_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

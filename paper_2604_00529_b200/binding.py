@@ -68,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
+    L.mxq_slice_scale_batched_static.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
+    L.mxq_slice_scale_batched_static.restype = i
     for name in ("mxq_quantize", "mxq_slice_scale", "mxq_dequantize", "mxq_fake_quant", "mxq_fake_quant_bwd",
                  "mxq_slice_scale_batched"):
         getattr(L, name).restype = i
@@ -188,3 +190,22 @@ def slice_scale_batched(items: Sequence[Tuple[torch.Tensor, torch.Tensor, int, t
         arr[k] = _Item(_dev(c, "codes"), _dev(s, "scales"), n, _dev(oc, "out_codes"), _dev(os_, "out_scales"))
     _check(L.mxq_slice_scale_batched(arr, len(items), block, FORMATS[src_fmt], FORMATS[dst_fmt], _stream(stream)),
            "mxq_slice_scale_batched")
+
+
+#: largest item count mxq_slice_scale_batched_static accepts (MXQ_STATIC_BATCH_MAX in include/mxq.h)
+STATIC_BATCH_MAX = 1024
+
+
+def slice_scale_batched_static(items: Sequence[Tuple[torch.Tensor, torch.Tensor, int, torch.Tensor, torch.Tensor]],
+                               src_fmt: str, dst_fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_slice_scale_batched_static: slice_scale_batched for callers that may not allocate device
+    memory (a process whose own pool owns all of HBM, or a loop that cannot afford the device-wide
+    stall of cudaMalloc).  The item table is a fixed array inside libmxq, so at most STATIC_BATCH_MAX
+    items fit, and calls that can overlap on the GPU must not share a device.  The marshalling here
+    builds one small ctypes array on the host and touches no torch allocator."""
+    L = load_library()
+    arr = (_Item * len(items))()
+    for k, (c, s, n, oc, os_) in enumerate(items):
+        arr[k] = _Item(_dev(c, "codes"), _dev(s, "scales"), n, _dev(oc, "out_codes"), _dev(os_, "out_scales"))
+    _check(L.mxq_slice_scale_batched_static(arr, len(items), block, FORMATS[src_fmt], FORMATS[dst_fmt],
+                                            _stream(stream)), "mxq_slice_scale_batched_static")

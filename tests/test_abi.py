@@ -72,12 +72,13 @@ def test_argument_checks_answer_on_the_host(L):
     bw = L.mxq_fake_quant_bwd
     assert bw(A, 1, 64, A, None) == OK                                       # in place: no launch
     assert bw(A, 1, 64, None, None) == E_NULL
-    for fn in (L.mxq_slice_scale_batched,):
+    for fn in (L.mxq_slice_scale_batched, L.mxq_slice_scale_batched_static):
         assert fn(None, 3, 32, F["int8"], F["int4"], None) == E_NULL
         assert fn(None, -1, 32, F["int8"], F["int4"], None) == E_SIZE
         assert fn(None, 0, 32, F["int8"], F["int4"], None) == OK
         assert fn(None, 3, 16, F["int8"], F["int4"], None) == E_BLOCK
         assert fn(None, 3, 32, F["int8"], F["e2m1"], None) == E_PAIR
+    assert L.mxq_slice_scale_batched_static(None, 1025, 32, F["int8"], F["int4"], None) == E_SIZE
 
 
 def test_binding_refuses_cpu_tensors():
