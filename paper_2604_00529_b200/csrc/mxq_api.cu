@@ -13,29 +13,13 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 
-struct DeviceInfo {
-    int sm_count = 0;
-};
-
 std::mutex g_mutex;
-DeviceInfo g_dev[kMaxDevices];
 
 int current_device()
 {
     int d = 0;
     if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) return -1;
     return d;
-}
-
-int sm_count(int dev)
-{
-    std::lock_guard<std::mutex> lock(g_mutex);
-    if (g_dev[dev].sm_count == 0) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
-        g_dev[dev].sm_count = n;
-    }
-    return g_dev[dev].sm_count;
 }
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -60,19 +44,6 @@ struct ItemTable {
 ItemTable g_table[kMaxDevices];
 
 }  // namespace
-
-int grid_for(const void* kernel, size_t ntiles)
-{
-    const int dev = current_device();
-    const int sms = dev >= 0 ? sm_count(dev) : 1;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm <= 0)
-        per_sm = 1;
-    const size_t wave = (size_t)sms * (size_t)per_sm;
-    const size_t need = (ntiles + kWarpsPerCta - 1) / kWarpsPerCta;
-    const size_t g = need < wave ? need : wave;
-    return (int)(g ? g : 1);
-}
 
 }  // namespace mxq
 

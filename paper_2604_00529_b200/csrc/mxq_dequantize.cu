@@ -6,17 +6,18 @@ namespace mxq {
 namespace {
 
 constexpr int kU = 1;
+constexpr int kThreads = 128;
 
 template <class F, class T>
 int run(const void* codes, const uint8_t* scales, size_t n, int block, void* dst, cudaStream_t stream)
 {
-    auto kern = dequantize_kernel<F, T, kU>;
+    auto kern = dequantize_kernel<F, T, kU, kThreads>;
     const size_t nunits = n / 32;
     const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
     int shift = 0, per_unit = 1;
     if (block == 16) per_unit = 2;
     else while ((32 << shift) < block) ++shift;
-    kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(static_cast<const uint8_t*>(codes), scales,
+    kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(static_cast<const uint8_t*>(codes), scales,
                                                                         nunits, shift, per_unit,
                                                                         static_cast<uint8_t*>(dst));
     return MXQ_CHECK_LAUNCH();

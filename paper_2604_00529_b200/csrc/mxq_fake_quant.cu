@@ -6,7 +6,8 @@
 namespace mxq {
 namespace {
 
-constexpr int kU = 2;
+constexpr int kU = 1;
+constexpr int kThreads = 128;
 
 template <class T, class F, int BLOCK, int MODE>
 int run(const void* src, size_t n, void* dst, cudaStream_t stream)
@@ -14,10 +15,10 @@ int run(const void* src, size_t n, void* dst, cudaStream_t stream)
     if constexpr (BLOCK < T::epl) {
         return MXQ_ERR_BLOCK;
     } else {
-        auto kern = fake_quant_kernel<T, F, BLOCK, MODE, kU>;
+        auto kern = fake_quant_kernel<T, F, BLOCK, MODE, kU, kThreads>;
         const size_t nunits = n / T::epl;
         const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
-        kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(
+        kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(
             static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(dst));
         return MXQ_CHECK_LAUNCH();
     }
@@ -59,10 +60,10 @@ int launch_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, 
 
 int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream)
 {
-    constexpr int U = 4;
-    auto kern = copy_kernel<U>;
+    constexpr int U = 1, kCopyThreads = 256;
+    auto kern = copy_kernel<U, kCopyThreads>;
     const size_t ntiles = (nbytes / 32 + 32 * U - 1) / (32 * U);
-    kern<<<grid_for((const void*)kern, ntiles ? ntiles : 1), kThreads, 0, stream>>>(
+    kern<<<grid_for_tiles(ntiles, kCopyThreads), kCopyThreads, 0, stream>>>(
         static_cast<const uint8_t*>(src), nbytes, static_cast<uint8_t*>(dst));
     return MXQ_CHECK_LAUNCH();
 }

@@ -1,6 +1,9 @@
 // The streaming kernels of libmxq.  Common shape: every lane owns a "unit" of 32 bytes of the
 // widest stream it touches (one 256-bit global access), a warp sweeps tiles of 32*U consecutive
-// units, and warps stride over the tiles of the tensor (persistent grid sized from the SM count).
+// units, and warps stride over the tiles of the tensor.  The launchers start one warp per tile
+// (many small CTAs that the hardware schedules as earlier ones retire, which keeps the loads of new
+// CTAs overlapped with the arithmetic and stores of older ones); the stride loop only matters
+// when the tile count exceeds the grid limit.
 //
 //   quantize / fake_quant : unit = 32 B of FP32/BF16 input (8 / 16 elements); a block of 32
 //                           elements spans 4 / 2 adjacent lanes, whose maxima meet by xor-shuffles.
@@ -20,8 +23,6 @@
 
 namespace mxq {
 
-constexpr int kThreads = 256;
-constexpr int kWarpsPerCta = kThreads / 32;
 
 template <int N, class Fn>
 __device__ __forceinline__ void static_for(Fn&& fn)
@@ -115,8 +116,8 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
     });
 }
 
-template <class T, class F, int BLOCK, int U>
-__global__ void __launch_bounds__(kThreads)
+template <class T, class F, int BLOCK, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes,
                 uint8_t* __restrict__ scales)
 {
@@ -125,8 +126,8 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
     constexpr int OB = T::epl * F::bits / 8;            // code bytes per lane unit
     constexpr int NW = code_words(T::epl, F::bits);
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
@@ -240,8 +241,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return d;
 }
 
-template <class T, class F, int BLOCK, int MODE, int U>
-__global__ void __launch_bounds__(kThreads)
+template <class T, class F, int BLOCK, int MODE, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may equal src
 {
     using A = Fmt<F::kind == KIND_INT ? MXQ_INT8 : MXQ_FP8_E4M3>;
@@ -251,8 +252,8 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
     constexpr int LPB = BLOCK / T::epl;
     static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
@@ -437,7 +438,7 @@ __device__ __forceinline__ uint8_t ss_scale_byte(uint32_t b, int de)
 
 // One tensor's worth of work for a warp-strided sweep; shared by the single-tensor and the
 // batched kernels.  `first`/`stride` are in tiles.
-template <class FH, class FL, int U>
+template <class FH, class FL, int U, int THREADS>
 __device__ __forceinline__ void slice_scale_sweep(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
                                                   size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
                                                   uint8_t* __restrict__ out_scales, size_t first, size_t stride)
@@ -477,14 +478,14 @@ __device__ __forceinline__ void slice_scale_sweep(const uint8_t* __restrict__ co
     }
 }
 
-template <class FH, class FL, int U>
-__global__ void __launch_bounds__(kThreads)
+template <class FH, class FL, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                    size_t nscales, uint8_t* __restrict__ out_codes, uint8_t* __restrict__ out_scales)
 {
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
-    slice_scale_sweep<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, warp, nwarps);
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
+    slice_scale_sweep<FH, FL, U, THREADS>(codes, scales, nunits, nscales, out_codes, out_scales, warp, nwarps);
 }
 
 // Device-side item of the batched conversion (one tensor), with its place in the flattened
@@ -499,23 +500,28 @@ struct SsDeviceItem {
     size_t tile_begin;     // first global tile index of this tensor
 };
 
-// All tensors in one launch: the tiles of every tensor are laid end to end and warps stride over
-// that global tile space, so small tensors do not leave SMs idle.
-template <class FH, class FL, int U>
-__global__ void __launch_bounds__(kThreads)
+// All tensors in one launch: the tiles of every tensor are laid end to end and every warp finds the
+// tensor its tile belongs to by a binary search of the item table, so small tensors do not leave
+// SMs idle.
+template <class FH, class FL, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, size_t total_tiles)
 {
     constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;
     constexpr int NWI = IB / 4, NWO = OB / 4;
     constexpr int de = FH::emax - FL::emax;
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
-    int it = 0;
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     for (size_t tile = warp; tile < total_tiles; tile += nwarps) {
-        // items are sorted by tile_begin and tile only grows: advance linearly
-        while (it + 1 < count && items[it + 1].tile_begin <= tile) ++it;
-        const SsDeviceItem t = items[it];
+        // items are sorted by tile_begin: the last one that starts at or before this tile owns it
+        int lo = 0, hi = count - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (items[mid].tile_begin <= tile) lo = mid;
+            else hi = mid - 1;
+        }
+        const SsDeviceItem t = items[lo];
         const size_t u0 = (tile - t.tile_begin) * (32 * U) + lane;
         uint32_t w[U][NWI];
         uint32_t sb[U];
@@ -544,16 +550,16 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
 // Reconstruction V^ = X P.  One lane = 32 codes.
 // ------------------------------------------------------------------------------------------
 
-template <class F, class T, int U>
-__global__ void __launch_bounds__(kThreads)
+template <class F, class T, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                   int units_per_scale_shift, int scales_per_unit, uint8_t* __restrict__ dst)
 {
     constexpr int IB = 4 * F::bits, NWI = IB / 4;
     constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
@@ -623,14 +629,14 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
 // Straight-through backward: a plain copy
 // ------------------------------------------------------------------------------------------
 
-template <int U>
-__global__ void __launch_bounds__(kThreads)
+template <int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict__ dst)
 {
     const size_t nunits = nbytes / 32;
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * kWarpsPerCta;
+    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
@@ -643,8 +649,8 @@ copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict_
             if (u0 + u * 32 < nunits) st256(dst + (u0 + u * 32) * 32, w[u]);
     }
     // ragged tail (n * size need not be a multiple of 32 bytes)
-    const size_t tid = (size_t)blockIdx.x * kThreads + threadIdx.x;
-    for (size_t i = nunits * 32 + tid; i < nbytes; i += (size_t)gridDim.x * kThreads) dst[i] = src[i];
+    const size_t tid = (size_t)blockIdx.x * THREADS + threadIdx.x;
+    for (size_t i = nunits * 32 + tid; i < nbytes; i += (size_t)gridDim.x * THREADS) dst[i] = src[i];
 }
 
 }  // namespace mxq

@@ -9,9 +9,15 @@
 
 namespace mxq {
 
-// Persistent-grid size for a kernel: enough CTAs for `ntiles` warp tiles, at most one full wave
-// (SM count x resident CTAs per SM for this kernel on the current device).
-int grid_for(const void* kernel, size_t ntiles);
+// Grid size that gives every warp tile a warp of its own (`threads` per CTA), capped at the largest
+// grid the kernels' stride loops are meant to cover.
+inline int grid_for_tiles(size_t ntiles, int threads)
+{
+    const size_t warps = (size_t)threads / 32;
+    const size_t need = (ntiles + warps - 1) / warps;
+    const size_t cap = (size_t)1 << 24;
+    return (int)(need < cap ? (need ? need : 1) : cap);
+}
 
 int launch_quantize(const void* src, int dtype, size_t n, int fmt, int block, void* codes, uint8_t* scales,
                     cudaStream_t stream);

@@ -6,7 +6,10 @@
 namespace mxq {
 namespace {
 
-constexpr int kU = 2;   // lane units in flight per thread
+// lane units in flight per thread: the MXINT quantizer is bound by its integer arithmetic and gains
+// from more independent work per thread; the MXFP one is bound by HBM alone
+template <class F> constexpr int kU = F::kind == KIND_INT ? 4 : 2;
+constexpr int kThreads = 128;
 
 template <class T, class F, int BLOCK>
 int run(const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t stream)
@@ -14,10 +17,11 @@ int run(const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t st
     if constexpr (BLOCK < T::epl) {
         return MXQ_ERR_BLOCK;
     } else {
-        auto kern = quantize_kernel<T, F, BLOCK, kU>;
+        constexpr int U = kU<F>;
+        auto kern = quantize_kernel<T, F, BLOCK, U, kThreads>;
         const size_t nunits = n / T::epl;
-        const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
-        kern<<<grid_for((const void*)kern, ntiles), kThreads, 0, stream>>>(
+        const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+        kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(
             static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(codes), scales);
         return MXQ_CHECK_LAUNCH();
     }
