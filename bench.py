@@ -8,7 +8,7 @@ BF16 8192 x 8192 weight matrix, Student-t with outliers): quantize to the MXFP8 
 MXINT8 anchors, Slice-and-Scale to MXFP6 (E2M3) / MXFP4 (E2M1) / MXINT6 / MXINT4, the same
 conversion through the batched entry point, reconstruction to BF16, the fused fake-quant
 forward through the anchor and its straight-through backward.  Consumers read what the
-*previous* step produced (two buffer sets), so no kernel finds its input in L2.
+*previous* step produced (four buffer sets, each with its own copy of the input), so no kernel finds its input in L2.
 
 Prints ONE JSON line on stdout: whole-step algorithmic GB/s (`value`), the end-to-end figure
 with host buffers (`e2e`), the roofline record of the dominant kernel, per-kernel figures,
@@ -152,19 +152,24 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------
 
 class HotPath:
-    """Device buffers and the op list of one step.  Two buffer sets: set j is written by the
-    producers of step j (mod 2) and read by the consumers of the following step."""
+    """Device buffers and the op list of one step.  NSETS buffer sets (each with its own copy of
+    the input tensor): set j is written by the producers of step j (mod NSETS) and read by the
+    consumers of the following step, so a buffer is touched again only after about NSETS x 0.9 GB
+    of other traffic has gone through the 126 MB L2."""
+
+    NSETS = 4
 
     def __init__(self, x_host_bits: np.ndarray, device):
         import torch
         import paper_2604_00529_b200 as mxq
         self.torch, self.mxq = torch, mxq
         self.n = n = int(x_host_bits.size)
-        self.x = torch.from_numpy(x_host_bits.view(np.int16)).to(device).view(torch.bfloat16)
+        x0 = torch.from_numpy(x_host_bits.view(np.int16)).to(device).view(torch.bfloat16)
+        self.xs = [x0] + [x0.clone() for _ in range(self.NSETS - 1)]
         u8 = dict(dtype=torch.uint8, device=device)
         nb = n // BLOCK
         self.sets = []
-        for _ in range(2):
+        for _ in range(self.NSETS):
             s = {}
             for name, bits in (("e4m3", 8), ("int8", 8), ("e2m3", 6), ("e2m1", 4), ("int6", 6), ("int4", 4),
                                ("e2m1_b", 4)):
@@ -176,8 +181,9 @@ class HotPath:
             self.sets.append(s)
         self.parts = 8                          # the batched entry point sees the tensor as 8 row bands
         self.op_names = list(OP_BYTES)
-        # item lists of the batched conversion: read set 1-j, write set j
-        self.items = [self.batched_items(self.sets[1 - j]["e4m3"], self.sets[j]["e2m1_b"]) for j in range(2)]
+        # item lists of the batched conversion: read set j-1, write set j
+        self.items = [self.batched_items(self.sets[(j - 1) % self.NSETS]["e4m3"], self.sets[j]["e2m1_b"])
+                      for j in range(self.NSETS)]
 
     def batched_items(self, src, dst):
         n, p = self.n, self.parts
@@ -188,23 +194,28 @@ class HotPath:
                           dst[0][k * m // 2:(k + 1) * m // 2], dst[1][k * m // BLOCK:(k + 1) * m // BLOCK]))
         return items
 
-    def step(self, i: int, mark=None):
-        """Runs the ops of step i; `mark(k)` is called before op k and after the last one."""
+    def step(self, i: int, mark=None, only=None):
+        """Runs the ops of step i (or just op `only`); `mark(k)` is called before op k and after
+        the last one."""
         mxq, n = self.mxq, self.n
-        cur, prev = self.sets[i & 1], self.sets[(i + 1) & 1]
+        j = i % self.NSETS
+        cur, prev, x = self.sets[j], self.sets[(j - 1) % self.NSETS], self.xs[j]
         ops = [
-            lambda: mxq.quantize(self.x, "e4m3", BLOCK, *cur["e4m3"]),
-            lambda: mxq.quantize(self.x, "int8", BLOCK, *cur["int8"]),
+            lambda: mxq.quantize(x, "e4m3", BLOCK, *cur["e4m3"]),
+            lambda: mxq.quantize(x, "int8", BLOCK, *cur["int8"]),
             lambda: mxq.slice_scale(*prev["e4m3"], n, "e4m3", "e2m3", BLOCK, *cur["e2m3"]),
             lambda: mxq.slice_scale(*prev["e4m3"], n, "e4m3", "e2m1", BLOCK, *cur["e2m1"]),
             lambda: mxq.slice_scale(*prev["int8"], n, "int8", "int6", BLOCK, *cur["int6"]),
             lambda: mxq.slice_scale(*prev["int8"], n, "int8", "int4", BLOCK, *cur["int4"]),
-            lambda: mxq.slice_scale_batched(self.items[i & 1], "e4m3", "e2m1", BLOCK),
+            lambda: mxq.slice_scale_batched(self.items[j], "e4m3", "e2m1", BLOCK),
             lambda: mxq.dequantize(*prev["e2m1"], n, "e2m1", BLOCK, dst=cur["deq_e2m1"]),
             lambda: mxq.dequantize(*prev["int4"], n, "int4", BLOCK, dst=cur["deq_int4"]),
-            lambda: mxq.fake_quant(self.x, "e2m3", BLOCK, mxq.FQ_VIA_ANCHOR, dst=cur["fq"]),
+            lambda: mxq.fake_quant(x, "e2m3", BLOCK, mxq.FQ_VIA_ANCHOR, dst=cur["fq"]),
             lambda: mxq.fake_quant_bwd(prev["fq"], cur["grad"]),
         ]
+        if only is not None:
+            ops[only]()
+            return 1
         for k, op in enumerate(ops):
             if mark:
                 mark(k)
@@ -260,7 +271,7 @@ def run_cuda(args):
     barrier()
 
     stream = torch.cuda.current_stream()
-    base = i + (i & 1)                      # keep the set parity continuous with the warm-up
+    base = i                                # continue the rotation of buffer sets where the warm-up stopped
     # timed region 1 -- the headline: K steps back to back between two events, nothing else in the stream
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -280,6 +291,20 @@ def run_cuda(args):
     barrier()
     op_ms = [sum(events[s][k].elapsed_time(events[s][k + 1]) for s in range(args.steps)) / args.steps
              for k in range(nops)]
+    # timed region 3 -- every op on its own: K launches of the same kernel back to back between two
+    # events, rotating over the buffer sets; this is the average launch duration the roofline uses
+    iso_ms = []
+    for k in range(nops):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for s in range(3):
+            hp.step(base + s, only=k)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for s in range(args.steps):
+            hp.step(base + s, only=k)
+        b.record(stream)
+        torch.cuda.synchronize()
+        iso_ms.append(a.elapsed_time(b) / args.steps)
     if world > 1:
         t = torch.tensor([total_ms], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -298,9 +323,9 @@ def run_cuda(args):
     d2h = sum(a.numel() + b.numel() for a, b in host_out.values())
 
     def e2e_step(i):
-        hp.x.view(torch.int16).copy_(host_in, non_blocking=True)
+        hp.xs[i % hp.NSETS].view(torch.int16).copy_(host_in, non_blocking=True)
         hp.step(i)
-        cur = hp.sets[i & 1]
+        cur = hp.sets[i % hp.NSETS]
         for k in outs:
             host_out[k][0].copy_(cur[k][0], non_blocking=True)
             host_out[k][1].copy_(cur[k][1], non_blocking=True)
@@ -328,13 +353,14 @@ def run_cuda(args):
     step_bytes = STEP_BYTES_PER_ELEM * n
     value = step_bytes * world / (ms_per_step * 1e-3) / 1e9
     per_op = {}
-    for name, ms in zip(hp.op_names, op_ms):
+    for name, ms, ms_in_step in zip(hp.op_names, iso_ms, op_ms):
         gbs = OP_BYTES[name] * n / (ms * 1e-3) / 1e9
-        per_op[name] = {"ms": round(ms, 5), "gbs": round(gbs, 1), "gelem_s": round(n / (ms * 1e-3) / 1e9, 2),
+        per_op[name] = {"ms": round(ms, 5), "ms_in_step_with_events": round(ms_in_step, 5), "gbs": round(gbs, 1),
+                        "gelem_s": round(n / (ms * 1e-3) / 1e9, 2),
                         "frac_of_%s_peak" % peak_kind: round(gbs / peak, 4), "frac_of_8000": round(gbs / 8000.0, 4)}
-    top = max(range(nops), key=lambda k: op_ms[k])
+    top = max(range(nops), key=lambda k: iso_ms[k])
     top_name = hp.op_names[top]
-    top_gbs = OP_BYTES[top_name] * n / (op_ms[top] * 1e-3) / 1e9
+    top_gbs = OP_BYTES[top_name] * n / (iso_ms[top] * 1e-3) / 1e9
     traffic = NCU_TRAFFIC.get(top_name) if kernel_sources_digest() == NCU_TRAFFIC_SOURCES else None
 
     cpu = cpu_baseline(x_bits)
@@ -345,8 +371,9 @@ def run_cuda(args):
         "data": "synthetic", "impl": "mxq",
         "config": {"workload": WORKLOAD, "elements_per_gpu": n, "block": BLOCK, "ops_per_step": hp.op_names,
                    "bytes_per_step_per_gpu": int(step_bytes), "l2": "inputs larger than L2; consumers read the "
-                   "previous step's buffers", "timing": "value: K steps between two events; kernels/roofline: a "
-                   "second pass of K steps with an event between launches", "gelem_per_s": round(n * nops * world / (ms_per_step * 1e-3) / 1e9, 2)},
+                   "previous step's buffers", "timing": "value: K steps between two events; kernels/roofline: K "
+                   "launches of one kernel back to back between two events, rotating over 4 buffer sets; "
+                   "ms_in_step_with_events: K steps with an event between launches", "gelem_per_s": round(n * nops * world / (ms_per_step * 1e-3) / 1e9, 2)},
         "e2e": {"value": round(step_bytes * world / (e2e_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                 "ms_per_step": round(e2e_ms, 4)},

@@ -7,6 +7,17 @@
 
 namespace mxq {
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization allowed: its
+// CTAs may become resident while the previous kernel of the stream is still draining, so the
+// ~2 us launch gap between short kernels disappears.  pdl_release() lets the next kernel start
+// launching; pdl_acquire() blocks until the previous kernel has completed and its writes are
+// visible.  Each kernel calls pdl_release() first and pdl_acquire() before its first global
+// memory access, which keeps plain stream-order semantics for every buffer.
+
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_acquire() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- 32-byte accesses ---------------------------------------------------------------------
 
 __device__ __forceinline__ void ld256(uint32_t (&w)[8], const void* p)

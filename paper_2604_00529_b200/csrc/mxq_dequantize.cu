@@ -17,10 +17,8 @@ int run(const void* codes, const uint8_t* scales, size_t n, int block, void* dst
     int shift = 0, per_unit = 1;
     if (block == 16) per_unit = 2;
     else while ((32 << shift) < block) ++shift;
-    kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(static_cast<const uint8_t*>(codes), scales,
-                                                                        nunits, shift, per_unit,
-                                                                        static_cast<uint8_t*>(dst));
-    return MXQ_CHECK_LAUNCH();
+    return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream, static_cast<const uint8_t*>(codes),
+                         scales, nunits, shift, per_unit, static_cast<uint8_t*>(dst));
 }
 
 }  // namespace

@@ -18,9 +18,8 @@ int run(const void* src, size_t n, void* dst, cudaStream_t stream)
         auto kern = fake_quant_kernel<T, F, BLOCK, MODE, kU, kThreads>;
         const size_t nunits = n / T::epl;
         const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
-        kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(
-            static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(dst));
-        return MXQ_CHECK_LAUNCH();
+        return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream,
+                             static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(dst));
     }
 }
 
@@ -63,9 +62,8 @@ int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream)
     constexpr int U = 1, kCopyThreads = 256;
     auto kern = copy_kernel<U, kCopyThreads>;
     const size_t ntiles = (nbytes / 32 + 32 * U - 1) / (32 * U);
-    kern<<<grid_for_tiles(ntiles, kCopyThreads), kCopyThreads, 0, stream>>>(
-        static_cast<const uint8_t*>(src), nbytes, static_cast<uint8_t*>(dst));
-    return MXQ_CHECK_LAUNCH();
+    return launch_kernel(kern, grid_for_tiles(ntiles, kCopyThreads), kCopyThreads, stream,
+                         static_cast<const uint8_t*>(src), nbytes, static_cast<uint8_t*>(dst));
 }
 
 }  // namespace mxq

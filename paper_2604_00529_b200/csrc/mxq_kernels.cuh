@@ -96,24 +96,109 @@ __device__ __forceinline__ uint32_t group_max(uint32_t v)
 // Q_f: quantize (Eq. 1-3)
 // ------------------------------------------------------------------------------------------
 
+// 4 bytes holding 6-bit codes -> 24-bit stream
+__device__ __forceinline__ uint32_t squeeze6(uint32_t x)
+{
+    uint32_t y = (x & 0x003F003Fu) | ((x & 0x3F003F00u) >> 2);
+    return (y & 0x00000FFFu) | ((y >> 4) & 0x00FFF000u);
+}
+
+// MXINT codes of four consecutive elements (Eq. 3), one per byte in the low F::bits bits.
+//   v0..v3 : the raw elements, inv = 2^-shared_exp (|v| inv < 2^(bits-1), exact)
+//   full   : 0xFF in the bytes whose element is negative, 0x00 elsewhere
+// One round-down FFMA per element adds 2^15 + 0.5, where the FP32 spacing is 2^-8: byte 1 of the
+// sum is floor(|r| + 0.5), the magnitude rounded to nearest with ties away from zero.  Three byte
+// permutes gather the four magnitudes; clip and sign are then applied to all four at once.
+template <class F>
+__device__ __forceinline__ uint32_t quantize_int_quad(float v0, float v1, float v2, float v3, float inv, uint32_t full)
+{
+    constexpr float kMagic = 32768.5f;
+    constexpr uint32_t k01 = 0x01010101u;
+    constexpr uint32_t kInv255 = 0xFEFEFEFFu;                  // 255^-1 mod 2^32: mask -> 0/1 per byte
+    constexpr uint32_t kMask = k01 * F::mask;
+    const uint32_t y0 = __float_as_uint(__fmaf_rd(fabsf(v0), inv, kMagic));
+    const uint32_t y1 = __float_as_uint(__fmaf_rd(fabsf(v1), inv, kMagic));
+    const uint32_t y2 = __float_as_uint(__fmaf_rd(fabsf(v2), inv, kMagic));
+    const uint32_t y3 = __float_as_uint(__fmaf_rd(fabsf(v3), inv, kMagic));
+    uint32_t q = __byte_perm(__byte_perm(y0, y1, 0x0051), __byte_perm(y2, y3, 0x0051), 0x5410);
+    q -= (q >> (F::bits - 1)) & k01;                           // 2^(b-1) -> 2^(b-1) - 1 (symmetric clip)
+    if constexpr (F::bits == 8) {
+        // negate in 7 bits, then set the sign bit: no carry leaves a byte even for a negative zero
+        const uint32_t z = (q ^ (full & 0x7F7F7F7Fu)) + full * kInv255;
+        return z ^ (full & 0x80808080u);
+    } else {
+        return ((q ^ (full & kMask)) + full * kInv255) & kMask;
+    }
+}
+
+// 0xFF / 0x00 per byte: the signs of elements 4Q .. 4Q+3 of a lane unit, straight from the raw words.
+template <class T, int Q>
+__device__ __forceinline__ uint32_t unit_sign_bytes(const uint32_t (&w)[8])
+{
+    uint32_t full;
+    if constexpr (T::size == 2) {
+        // two BF16 per word: sign bits sit at the top of bytes 1 and 3 (selector bit 3 replicates it)
+        asm("prmt.b32 %0, %1, %2, 0xFDB9;" : "=r"(full) : "r"(w[2 * Q]), "r"(w[2 * Q + 1]));
+    } else {
+        uint32_t a, b;
+        asm("prmt.b32 %0, %1, %2, 0x00FB;" : "=r"(a) : "r"(w[4 * Q]), "r"(w[4 * Q + 1]));
+        asm("prmt.b32 %0, %1, %2, 0x00FB;" : "=r"(b) : "r"(w[4 * Q + 2]), "r"(w[4 * Q + 3]));
+        full = __byte_perm(a, b, 0x5410);
+    }
+    return full;
+}
+
 // Codes of one lane unit, packed as a little-endian bitstream.
 template <class T, class F, int NW>
 __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv, uint32_t (&out)[NW])
 {
-    static_for<T::epl / 2>([&](auto i) {
-        constexpr int I = decltype(i)::value;
-        uint2 c = quantize_pair<F>(unit_elem<T, 2 * I>(w), unit_elem<T, 2 * I + 1>(w), inv);
+    if constexpr (F::kind == KIND_INT) {
+        constexpr int NQ = T::epl / 4;
+        uint32_t z[NQ];
+        static_for<NQ>([&](auto qi) {
+            constexpr int Q = decltype(qi)::value;
+            z[Q] = quantize_int_quad<F>(unit_elem<T, 4 * Q>(w), unit_elem<T, 4 * Q + 1>(w), unit_elem<T, 4 * Q + 2>(w),
+                                        unit_elem<T, 4 * Q + 3>(w), inv, unit_sign_bytes<T, Q>(w));
+        });
         if constexpr (F::bits == 8) {
-            // two bytes at a time
-            constexpr int wi = I / 2, sh = (I & 1) * 16;
-            uint32_t pair = c.x | (c.y << 8);
-            if constexpr (sh == 0) out[wi] = pair;
-            else out[wi] |= pair << 16;
+#pragma unroll
+            for (int j = 0; j < NQ; ++j) out[j] = z[j];
+        } else if constexpr (F::bits == 4) {
+            // c0 | c1 << 4 lands in byte 0 and c2 | c3 << 4 in byte 2 of z | z >> 4
+#pragma unroll
+            for (int j = 0; j < NQ / 2; ++j)
+                out[j] = __byte_perm(z[2 * j] | (z[2 * j] >> 4), z[2 * j + 1] | (z[2 * j + 1] >> 4), 0x6420);
+        } else if constexpr (F::bits == 6 && NQ % 4 == 0) {
+#pragma unroll
+            for (int g = 0; g < NQ / 4; ++g) {
+                const uint32_t s0 = squeeze6(z[4 * g]), s1 = squeeze6(z[4 * g + 1]), s2 = squeeze6(z[4 * g + 2]),
+                               s3 = squeeze6(z[4 * g + 3]);
+                out[3 * g + 0] = s0 | (s1 << 24);
+                out[3 * g + 1] = (s1 >> 8) | (s2 << 16);
+                out[3 * g + 2] = (s2 >> 16) | (s3 << 8);
+            }
         } else {
-            put_code<F::bits, 2 * I>(out, c.x);
-            put_code<F::bits, 2 * I + 1>(out, c.y);
+            static_for<T::epl>([&](auto i) {
+                constexpr int I = decltype(i)::value;
+                put_code<F::bits, I>(out, (z[I / 4] >> (8 * (I % 4))) & F::mask);
+            });
         }
-    });
+    } else {
+        static_for<T::epl / 2>([&](auto i) {
+            constexpr int I = decltype(i)::value;
+            uint2 c = quantize_pair<F>(unit_elem<T, 2 * I>(w), unit_elem<T, 2 * I + 1>(w), inv);
+            if constexpr (F::bits == 8) {
+                // two bytes at a time
+                constexpr int wi = I / 2, sh = (I & 1) * 16;
+                uint32_t pair = c.x | (c.y << 8);
+                if constexpr (sh == 0) out[wi] = pair;
+                else out[wi] |= pair << 16;
+            } else {
+                put_code<F::bits, 2 * I>(out, c.x);
+                put_code<F::bits, 2 * I + 1>(out, c.y);
+            }
+        });
+    }
 }
 
 template <class T, class F, int BLOCK, int U, int THREADS>
@@ -121,6 +206,7 @@ __global__ void __launch_bounds__(THREADS)
 quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes,
                 uint8_t* __restrict__ scales)
 {
+    pdl_release();
     constexpr int LPB = BLOCK / T::epl;                 // lanes per block
     static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
     constexpr int OB = T::epl * F::bits / 8;            // code bytes per lane unit
@@ -130,6 +216,7 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
+    pdl_acquire();
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];
@@ -245,6 +332,7 @@ template <class T, class F, int BLOCK, int MODE, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may equal src
 {
+    pdl_release();
     using A = Fmt<F::kind == KIND_INT ? MXQ_INT8 : MXQ_FP8_E4M3>;
     constexpr bool via = MODE == MXQ_FQ_VIA_ANCHOR && F::id != A::id;
     using S = std::conditional_t<via, A, F>;            // the format whose scale Eq. 1 computes
@@ -256,6 +344,7 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
+    pdl_acquire();
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];
@@ -310,30 +399,26 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
 // ------------------------------------------------------------------------------------------
 
 // Eq. 4 on four MXINT8 codes at once (one per byte): returns the four low-format codes, one per
-// byte, in the low BL bits.  Sign-magnitude SWAR; no carry ever crosses a byte.
+// byte, in the low BL bits.  Sign-magnitude SWAR; no carry ever crosses a byte.  The integer/logic
+// pipe is the scarce resource here, so the two places that need the per-byte sign as a 0/1 value
+// take it from the 0xFF/0x00 mask by one multiply-add with 255^-1 (mod 2^32), which runs on the
+// multiply pipe: mask = 255 * sum(s_i 256^i), hence mask * 255^-1 = sum(s_i 256^i) exactly.
 template <int BL>
 __device__ __forceinline__ uint32_t ss_int8_word(uint32_t x)
 {
     constexpr int de = 8 - BL;
     constexpr uint32_t k01 = 0x01010101u;
+    constexpr uint32_t kInv255 = 0xFEFEFEFFu;
     constexpr uint32_t kH = k01 * (1u << (de - 1));            // rounding increment
     constexpr uint32_t kLow = k01 * (0xFFu >> de);
     constexpr uint32_t kMask = k01 * ((1u << BL) - 1u);
     uint32_t full;                                            // 0xFF in the bytes that are negative
     asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(x));  // selector bit 3: replicate the byte's sign
-    uint32_t s1 = full & k01;
-    uint32_t a = x ^ full;                                     // |p| - s1
-    uint32_t t = a + s1 + kH;                                  // |p| + 2^(de-1) <= 160
-    uint32_t q = (t >> de) & kLow;                             // <= 2^(BL-1)
-    q -= (q >> (BL - 1)) & k01;                                // clip to 2^(BL-1) - 1
-    return ((q ^ (full & kMask)) + s1) & kMask;                // two's complement in BL bits
-}
-
-// 4 bytes holding 6-bit codes -> 24-bit stream
-__device__ __forceinline__ uint32_t squeeze6(uint32_t x)
-{
-    uint32_t y = (x & 0x003F003Fu) | ((x & 0x3F003F00u) >> 2);
-    return (y & 0x00000FFFu) | ((y >> 4) & 0x00FFF000u);
+    const uint32_t a = x ^ full;                               // |p| - s
+    const uint32_t t = a + full * kInv255 + kH;                // |p| + 2^(de-1) <= 127 + 64
+    const uint32_t c = (t >> 7) & k01;                         // 1 where the shifted value would be 2^(BL-1)
+    const uint32_t q = ((t >> de) & kLow) - c;                 // clipped to 2^(BL-1) - 1
+    return (full * kInv255 + (q ^ (full & kMask))) & kMask;    // two's complement in BL bits
 }
 
 __device__ __forceinline__ bool has_e4m3_nan(uint32_t x)
@@ -483,8 +568,10 @@ __global__ void __launch_bounds__(THREADS)
 slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                    size_t nscales, uint8_t* __restrict__ out_codes, uint8_t* __restrict__ out_scales)
 {
+    pdl_release();
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
+    pdl_acquire();
     slice_scale_sweep<FH, FL, U, THREADS>(codes, scales, nunits, nscales, out_codes, out_scales, warp, nwarps);
 }
 
@@ -507,12 +594,14 @@ template <class FH, class FL, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, size_t total_tiles)
 {
+    pdl_release();
     constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;
     constexpr int NWI = IB / 4, NWO = OB / 4;
     constexpr int de = FH::emax - FL::emax;
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
+    pdl_acquire();
     for (size_t tile = warp; tile < total_tiles; tile += nwarps) {
         // items are sorted by tile_begin: the last one that starts at or before this tile owns it
         int lo = 0, hi = count - 1;
@@ -555,12 +644,14 @@ __global__ void __launch_bounds__(THREADS)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                   int units_per_scale_shift, int scales_per_unit, uint8_t* __restrict__ dst)
 {
+    pdl_release();
     constexpr int IB = 4 * F::bits, NWI = IB / 4;
     constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    pdl_acquire();
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][NWI];
@@ -633,11 +724,13 @@ template <int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict__ dst)
 {
+    pdl_release();
     const size_t nunits = nbytes / 32;
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    pdl_acquire();
     for (size_t tile = warp; tile < ntiles; tile += nwarps) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];

@@ -56,6 +56,26 @@ size_t ss_batched_tiles(size_t nunits);
     }
 #define MXQ_DISPATCH_FORMAT(fmt, ...) MXQ_DISPATCH_FORMAT_AS(fmt, F, __VA_ARGS__)
 
-#define MXQ_CHECK_LAUNCH() (cudaGetLastError() == cudaSuccess ? MXQ_OK : MXQ_ERR_CUDA)
+// Launches `kern` on `stream` with programmatic stream serialization allowed (see pdl_release /
+// pdl_acquire in mxq_access.cuh).  Returns MXQ_OK or MXQ_ERR_CUDA.
+template <class... KArgs, class... Args>
+inline int launch_kernel(void (*kern)(KArgs...), int grid, int threads, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    return MXQ_OK;
+}
 
 }  // namespace mxq

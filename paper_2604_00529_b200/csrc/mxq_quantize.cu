@@ -21,9 +21,8 @@ int run(const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t st
         auto kern = quantize_kernel<T, F, BLOCK, U, kThreads>;
         const size_t nunits = n / T::epl;
         const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
-        kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(
-            static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(codes), scales);
-        return MXQ_CHECK_LAUNCH();
+        return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream,
+                             static_cast<const uint8_t*>(src), nunits, static_cast<uint8_t*>(codes), scales);
     }
 }
 

@@ -22,10 +22,9 @@ int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int b
                 auto kern = slice_scale_kernel<FH, FL, kU, kThreads>;
                 const size_t nunits = n / 32, nscales = n / (size_t)block;
                 const size_t ntiles = ss_batched_tiles(nunits);
-                kern<<<grid_for_tiles(ntiles, kThreads), kThreads, 0, stream>>>(
-                    static_cast<const uint8_t*>(codes), scales, nunits, nscales, static_cast<uint8_t*>(out_codes),
-                    out_scales);
-                return MXQ_CHECK_LAUNCH();
+                return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream,
+                                     static_cast<const uint8_t*>(codes), scales, nunits, nscales,
+                                     static_cast<uint8_t*>(out_codes), out_scales);
             } else {
                 return MXQ_ERR_PAIR;
             }
@@ -41,8 +40,8 @@ int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t 
         MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, {
             if constexpr (ss_pair_ok(FH::id, FL::id)) {
                 auto kern = slice_scale_batched_kernel<FH, FL, kU, kThreads>;
-                kern<<<grid_for_tiles(total_tiles, kThreads), kThreads, 0, stream>>>(items_dev, count, total_tiles);
-                return MXQ_CHECK_LAUNCH();
+                return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, items_dev, count,
+                                     total_tiles);
             } else {
                 return MXQ_ERR_PAIR;
             }
