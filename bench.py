@@ -293,16 +293,18 @@ def run_cuda(args):
              for k in range(nops)]
     # timed region 3 -- every op on its own: K launches of the same kernel back to back between two
     # events, rotating over the buffer sets; this is the average launch duration the roofline uses
-    iso_ms = []
+    iso_ms, host_ms = [], []
     for k in range(nops):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for s in range(3):
             hp.step(base + s, only=k)
         torch.cuda.synchronize()
+        h0 = time.perf_counter()
         a.record(stream)
         for s in range(args.steps):
             hp.step(base + s, only=k)
         b.record(stream)
+        host_ms.append((time.perf_counter() - h0) * 1e3 / args.steps)   # host time to enqueue one launch
         torch.cuda.synchronize()
         iso_ms.append(a.elapsed_time(b) / args.steps)
     if world > 1:
@@ -353,9 +355,10 @@ def run_cuda(args):
     step_bytes = STEP_BYTES_PER_ELEM * n
     value = step_bytes * world / (ms_per_step * 1e-3) / 1e9
     per_op = {}
-    for name, ms, ms_in_step in zip(hp.op_names, iso_ms, op_ms):
+    for name, ms, ms_in_step, ms_host in zip(hp.op_names, iso_ms, op_ms, host_ms):
         gbs = OP_BYTES[name] * n / (ms * 1e-3) / 1e9
-        per_op[name] = {"ms": round(ms, 5), "ms_in_step_with_events": round(ms_in_step, 5), "gbs": round(gbs, 1),
+        per_op[name] = {"ms": round(ms, 5), "ms_in_step_with_events": round(ms_in_step, 5),
+                        "host_enqueue_ms": round(ms_host, 5), "gbs": round(gbs, 1),
                         "gelem_s": round(n / (ms * 1e-3) / 1e9, 2),
                         "frac_of_%s_peak" % peak_kind: round(gbs / peak, 4), "frac_of_8000": round(gbs / 8000.0, 4)}
     top = max(range(nops), key=lambda k: iso_ms[k])

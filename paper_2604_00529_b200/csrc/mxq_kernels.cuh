@@ -1,9 +1,8 @@
 // The streaming kernels of libmxq.  Common shape: every lane owns a "unit" of 32 bytes of the
 // widest stream it touches (one 256-bit global access), a warp sweeps tiles of 32*U consecutive
-// units, and warps stride over the tiles of the tensor.  The launchers start one warp per tile
-// (many small CTAs that the hardware schedules as earlier ones retire, which keeps the loads of new
-// CTAs overlapped with the arithmetic and stores of older ones); the stride loop only matters
-// when the tile count exceeds the grid limit.
+// units, and every tile gets a warp of its own: many small CTAs that the hardware schedules as
+// earlier ones retire, which keeps the loads of new CTAs overlapped with the arithmetic and stores
+// of older ones (a persistent wave with a stride loop measured 10-20 % slower on these streams).
 //
 //   quantize / fake_quant : unit = 32 B of FP32/BF16 input (8 / 16 elements); a block of 32
 //                           elements spans 4 / 2 adjacent lanes, whose maxima meet by xor-shuffles.
@@ -213,11 +212,10 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
     constexpr int NW = code_words(T::epl, F::bits);
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
     pdl_acquire();
-    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+    if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];
 #pragma unroll
@@ -341,11 +339,10 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
     static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
 
     pdl_acquire();
-    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+    if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];
 #pragma unroll
@@ -521,45 +518,44 @@ __device__ __forceinline__ uint8_t ss_scale_byte(uint32_t b, int de)
     return (uint8_t)(b == 0xFFu ? 0xFFu : min(b + (uint32_t)de, 254u));
 }
 
-// One tensor's worth of work for a warp-strided sweep; shared by the single-tensor and the
-// batched kernels.  `first`/`stride` are in tiles.
-template <class FH, class FL, int U, int THREADS>
-__device__ __forceinline__ void slice_scale_sweep(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
-                                                  size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
-                                                  uint8_t* __restrict__ out_scales, size_t first, size_t stride)
+// One warp tile (32 U lane units) of one tensor; shared by the single-tensor and the batched
+// kernels.  The scale bytes are an element-wise stream of their own: lane unit i also converts
+// scale i, and scale nunits + i when the block is smaller than a lane unit (block 16).
+template <class FH, class FL, int U>
+__device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                 size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
+                                                 uint8_t* __restrict__ out_scales, size_t tile)
 {
     constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;      // bytes per lane unit
     constexpr int NWI = IB / 4, NWO = OB / 4;
     constexpr int de = FH::emax - FL::emax;
-    const int lane = threadIdx.x & 31;
-    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
-    for (size_t tile = first; tile < ntiles; tile += stride) {
-        const size_t u0 = tile * (32 * U) + lane;
-        uint32_t w[U][NWI];
-        uint32_t sb[U];
+    const size_t u0 = tile * (32 * U) + (threadIdx.x & 31);
+    uint32_t w[U][NWI];
+    uint32_t sb[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
-            else {
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
+        else {
 #pragma unroll
-                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
-            }
-            sb[u] = unit < nscales ? scales[unit] : 0;
+            for (int j = 0; j < NWI; ++j) w[u][j] = 0;
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            uint32_t out[NWO];
-            slice_scale_unit<FH, FL>(w[u], out);
-            if (unit < nunits) store_bytes<OB>(out_codes + unit * OB, out);
-            if (unit < nscales) out_scales[unit] = ss_scale_byte(sb[u], de);
-        }
+        sb[u] = unit < nscales ? scales[unit] : 0;
     }
-    // scale entries beyond the number of code units (block < 32): leftover element-wise pass
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit < nscales) out_scales[unit] = ss_scale_byte(sb[u], de);
+        uint32_t out[NWO];
+        slice_scale_unit<FH, FL>(w[u], out);
+        if (unit < nunits) store_bytes<OB>(out_codes + unit * OB, out);
+    }
     if (nscales > nunits) {
-        const size_t tid = first * 32 + lane, nthreads = stride * 32;
-        for (size_t i = nunits + tid; i < nscales; i += nthreads) out_scales[i] = ss_scale_byte(scales[i], de);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t i = nunits + u0 + u * 32;
+            if (i < nscales) out_scales[i] = ss_scale_byte(scales[i], de);
+        }
     }
 }
 
@@ -569,10 +565,9 @@ slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
                    size_t nscales, uint8_t* __restrict__ out_codes, uint8_t* __restrict__ out_scales)
 {
     pdl_release();
-    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     pdl_acquire();
-    slice_scale_sweep<FH, FL, U, THREADS>(codes, scales, nunits, nscales, out_codes, out_scales, warp, nwarps);
+    if (tile * (32 * U) < nunits) slice_scale_tile<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, tile);
 }
 
 // Device-side item of the batched conversion (one tensor), with its place in the flattened
@@ -595,44 +590,18 @@ __global__ void __launch_bounds__(THREADS)
 slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, size_t total_tiles)
 {
     pdl_release();
-    constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;
-    constexpr int NWI = IB / 4, NWO = OB / 4;
-    constexpr int de = FH::emax - FL::emax;
-    const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     pdl_acquire();
-    for (size_t tile = warp; tile < total_tiles; tile += nwarps) {
-        // items are sorted by tile_begin: the last one that starts at or before this tile owns it
-        int lo = 0, hi = count - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (items[mid].tile_begin <= tile) lo = mid;
-            else hi = mid - 1;
-        }
-        const SsDeviceItem t = items[lo];
-        const size_t u0 = (tile - t.tile_begin) * (32 * U) + lane;
-        uint32_t w[U][NWI];
-        uint32_t sb[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit < t.nunits) load_words<NWI>(w[u], t.codes + unit * IB);
-            else {
-#pragma unroll
-                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
-            }
-            sb[u] = unit < t.nscales ? t.scales[unit] : 0;
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            uint32_t out[NWO];
-            slice_scale_unit<FH, FL>(w[u], out);
-            if (unit < t.nunits) store_bytes<OB>(t.out_codes + unit * OB, out);
-            if (unit < t.nscales) t.out_scales[unit] = ss_scale_byte(sb[u], de);
-        }
+    if (tile >= total_tiles) return;
+    // items are sorted by tile_begin: the last one that starts at or before this tile owns it
+    int lo = 0, hi = count - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (items[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
     }
+    const SsDeviceItem t = items[lo];
+    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -649,10 +618,9 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
     pdl_acquire();
-    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+    if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][NWI];
 #pragma unroll
@@ -728,10 +696,9 @@ copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict_
     const size_t nunits = nbytes / 32;
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t nwarps = (size_t)gridDim.x * (THREADS / 32);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
     pdl_acquire();
-    for (size_t tile = warp; tile < ntiles; tile += nwarps) {
+    if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
         uint32_t w[U][8];
 #pragma unroll

@@ -9,14 +9,14 @@
 
 namespace mxq {
 
-// Grid size that gives every warp tile a warp of its own (`threads` per CTA), capped at the largest
-// grid the kernels' stride loops are meant to cover.
+// Grid size that gives every warp tile a warp of its own (`threads` per CTA); 0 when the tensor
+// would need more CTAs than a grid can hold (beyond 2^40 elements: reported as MXQ_ERR_SIZE).
 inline int grid_for_tiles(size_t ntiles, int threads)
 {
     const size_t warps = (size_t)threads / 32;
     const size_t need = (ntiles + warps - 1) / warps;
-    const size_t cap = (size_t)1 << 24;
-    return (int)(need < cap ? (need ? need : 1) : cap);
+    if (need > (size_t)0x7FFFFFFF) return 0;
+    return (int)(need ? need : 1);
 }
 
 int launch_quantize(const void* src, int dtype, size_t n, int fmt, int block, void* codes, uint8_t* scales,
@@ -61,6 +61,7 @@ size_t ss_batched_tiles(size_t nunits);
 template <class... KArgs, class... Args>
 inline int launch_kernel(void (*kern)(KArgs...), int grid, int threads, cudaStream_t stream, Args... args)
 {
+    if (grid <= 0) return MXQ_ERR_SIZE;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)threads);
