@@ -159,8 +159,9 @@ class HotPath:
 
     NSETS = 4
 
-    def __init__(self, x_host_bits: np.ndarray, device):
+    def __init__(self, x_host_bits: np.ndarray, device, nsets: int = 4):
         import torch
+        self.NSETS = nsets
         import paper_2604_00529_b200 as mxq
         self.torch, self.mxq = torch, mxq
         self.n = n = int(x_host_bits.size)
@@ -182,7 +183,7 @@ class HotPath:
         self.parts = 8                          # the batched entry point sees the tensor as 8 row bands
         self.op_names = list(OP_BYTES)
         # item lists of the batched conversion: read set j-1, write set j
-        self.items = [self.batched_items(self.sets[(j - 1) % self.NSETS]["e4m3"], self.sets[j]["e2m1_b"])
+        self.items = [mxq.make_items(self.batched_items(self.sets[(j - 1) % self.NSETS]["e4m3"], self.sets[j]["e2m1_b"]))
                       for j in range(self.NSETS)]
 
     def batched_items(self, src, dst):
@@ -245,7 +246,7 @@ def run_cuda(args):
     # weak scaling: every rank converts its own tensor of the workload's shape (blocks are
     # independent, so ranks exchange nothing); seed 1 on rank 0 is the documented workload
     x_bits = inputs.weight_bf16_student_t(ROWS, COLS, seed=1 + rank)
-    hp = HotPath(x_bits, device)
+    hp = HotPath(x_bits, device, args.buffer_sets)
     n = hp.n
     nops = len(hp.op_names)
 
@@ -464,8 +465,11 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="mxq", choices=["mxq", "reference"])
+    ap.add_argument("--buffer-sets", type=int, default=4,
+                    help="rotating buffer sets (>= 2); profiling captures use 2 to hold less device memory")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.buffer_sets = max(args.buffer_sets, 2)
     if args.impl == "reference":
         run_reference(args)
     else:

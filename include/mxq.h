@@ -146,11 +146,12 @@ int mxq_fake_quant_bwd(const void *grad_out, int dtype, size_t n, void *grad_in,
 /*
  * Whole-model on-the-fly conversion (Sec. 3.5, Inference): mxq_slice_scale over `count`
  * tensors in one launch.  `items` is a HOST array; every pointer inside is a device
- * pointer with the same requirements as in mxq_slice_scale.  The item table is copied to
- * a device-side table owned by the library (grown with cudaMalloc on first use or when
- * `count` exceeds its capacity, reused afterwards); the host array may be freed as soon
- * as the call returns.  Calls that share the table are ordered by `stream`; concurrent
- * calls on different streams are not supported.
+ * pointer with the same requirements as in mxq_slice_scale; the host array may be freed
+ * as soon as the call returns.  Up to 512 non-empty tensors travel in the kernel's own
+ * parameter space (no allocation, no copy).  Beyond that the item table is copied to a
+ * device-side table owned by the library (grown with cudaMalloc on first use or when
+ * `count` exceeds its capacity, reused afterwards); such calls are ordered by `stream`
+ * and must not run concurrently on different streams.
  */
 typedef struct {
     const void *codes;

@@ -181,15 +181,32 @@ def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = Non
     return grad_in
 
 
-def slice_scale_batched(items: Sequence[Tuple[torch.Tensor, torch.Tensor, int, torch.Tensor, torch.Tensor]],
-                        src_fmt: str, dst_fmt: str, block: int = 32, stream=None) -> None:
-    """mxq_slice_scale_batched over (codes, scales, n, out_codes, out_scales) tuples."""
+class ItemTable:
+    """A marshalled mxq_ss_item array: build it once with ``make_items`` for buffers that persist and
+    pass it to ``slice_scale_batched`` as often as needed (it keeps the tensors alive)."""
+
+    def __init__(self, items):
+        self.tensors = list(items)
+        self.array = (_Item * len(self.tensors))()
+        for k, (c, s, n, oc, os_) in enumerate(self.tensors):
+            self.array[k] = _Item(_dev(c, "codes"), _dev(s, "scales"), n, _dev(oc, "out_codes"), _dev(os_, "out_scales"))
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_items(items: Sequence[Tuple[torch.Tensor, torch.Tensor, int, torch.Tensor, torch.Tensor]]) -> ItemTable:
+    """Marshal (codes, scales, n, out_codes, out_scales) tuples into an mxq_ss_item array."""
+    return ItemTable(items)
+
+
+def slice_scale_batched(items, src_fmt: str, dst_fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_slice_scale_batched over (codes, scales, n, out_codes, out_scales) tuples, or over an
+    ItemTable made from them."""
     L = load_library()
-    arr = (_Item * len(items))()
-    for k, (c, s, n, oc, os_) in enumerate(items):
-        arr[k] = _Item(_dev(c, "codes"), _dev(s, "scales"), n, _dev(oc, "out_codes"), _dev(os_, "out_scales"))
-    _check(L.mxq_slice_scale_batched(arr, len(items), block, FORMATS[src_fmt], FORMATS[dst_fmt], _stream(stream)),
-           "mxq_slice_scale_batched")
+    table = items if isinstance(items, ItemTable) else ItemTable(items)
+    _check(L.mxq_slice_scale_batched(table.array, len(table), block, FORMATS[src_fmt], FORMATS[dst_fmt],
+                                     _stream(stream)), "mxq_slice_scale_batched")
 
 
 #: largest item count mxq_slice_scale_batched_static accepts (MXQ_STATIC_BATCH_MAX in include/mxq.h)

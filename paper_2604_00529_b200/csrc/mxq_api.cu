@@ -170,9 +170,12 @@ int mxq_slice_scale_batched(const mxq_ss_item* items, int count, int block, int 
     }
     if (host.empty()) return MXQ_OK;
 
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // up to kSsParamItemsMax tensors travel in the kernel's parameter space: nothing to allocate or copy
+    if ((int)host.size() <= kSsParamItemsMax)
+        return launch_slice_scale_batched_params(host.data(), (int)host.size(), tiles, src_fmt, dst_fmt, s);
     const int dev = current_device();
     if (dev < 0) return MXQ_ERR_CUDA;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     SsDeviceItem* table = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mutex);

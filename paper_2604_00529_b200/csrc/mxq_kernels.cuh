@@ -604,6 +604,32 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
     slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin);
 }
 
+// The same launch with the item table carried in the kernel's parameter space (K items, 56 bytes
+// each: K = 64 stays under the classic 4 KB of parameters, K = 512 uses the 32 KB that sm_70 and
+// later allow).  No device buffer, no host-to-device copy in front of the kernel.
+template <int K>
+struct SsItemBlock {
+    SsDeviceItem items[K];
+};
+
+template <class FH, class FL, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS)
+slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int count, size_t total_tiles)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    pdl_acquire();
+    if (tile >= total_tiles) return;
+    int lo = 0, hi = count - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (blk.items[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
+    }
+    const SsDeviceItem& t = blk.items[lo];
+    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin);
+}
+
 // ------------------------------------------------------------------------------------------
 // Reconstruction V^ = X P.  One lane = 32 codes.
 // ------------------------------------------------------------------------------------------

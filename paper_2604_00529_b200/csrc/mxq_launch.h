@@ -33,6 +33,11 @@ int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
 struct SsDeviceItem;
 int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t total_tiles, int src_fmt,
                                int dst_fmt, cudaStream_t stream);
+// The same launch with the items (a HOST array here) passed in the kernel's parameter space; count
+// must not exceed kSsParamItemsMax.
+constexpr int kSsParamItemsMax = 512;
+int launch_slice_scale_batched_params(const SsDeviceItem* items_host, int count, size_t total_tiles, int src_fmt,
+                                      int dst_fmt, cudaStream_t stream);
 // tiles one tensor of `nunits` lane units occupies in the batched kernel's tile space
 size_t ss_batched_tiles(size_t nunits);
 

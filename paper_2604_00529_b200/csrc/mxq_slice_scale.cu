@@ -50,4 +50,35 @@ int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t 
     return MXQ_ERR_FORMAT;
 }
 
+namespace {
+
+template <class FH, class FL, int K>
+int run_params(const SsDeviceItem* items_host, int count, size_t total_tiles, cudaStream_t stream)
+{
+    SsItemBlock<K> blk;
+    for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
+    for (int i = count; i < K; ++i) blk.items[i] = SsDeviceItem{};
+    auto kern = slice_scale_batched_param_kernel<FH, FL, kU, kThreads, K>;
+    return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
+}
+
+}  // namespace
+
+int launch_slice_scale_batched_params(const SsDeviceItem* items_host, int count, size_t total_tiles, int src_fmt,
+                                      int dst_fmt, cudaStream_t stream)
+{
+    if (count > kSsParamItemsMax) return MXQ_ERR_SIZE;
+    MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, {
+            if constexpr (ss_pair_ok(FH::id, FL::id)) {
+                if (count <= 64) return run_params<FH, FL, 64>(items_host, count, total_tiles, stream);
+                return run_params<FH, FL, kSsParamItemsMax>(items_host, count, total_tiles, stream);
+            } else {
+                return MXQ_ERR_PAIR;
+            }
+        });
+    });
+    return MXQ_ERR_FORMAT;
+}
+
 }  // namespace mxq

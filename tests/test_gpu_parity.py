@@ -183,6 +183,40 @@ def test_slice_scale_batched_matches_oracle():
             assert np.all(to_host(oc[nb:]) == 0xA5) and np.all(to_host(os_[n // 32:]) == 0xA5)
 
 
+@pytest.mark.parametrize("count", [64, 65, 512, 513, 700])
+def test_slice_scale_batched_item_counts(count):
+    """Item counts on both sides of the limits where the item table changes its way to the kernel
+    (small and large kernel-parameter blocks, device-side table)."""
+    rng = np.random.default_rng(count)
+    sizes = (64 * rng.integers(1, 8, count)).tolist()          # 64-element multiples keep every pointer 32-byte aligned
+    total = int(sum(sizes))
+    codes = rng.integers(0, 256, total).astype(np.uint8)
+    scales = rng.integers(0, 256, total // 32).astype(np.uint8)
+    # one arena per stream, tensors at 32-byte aligned offsets inside it
+    d_codes, d_scales = to_dev(codes), to_dev(np.repeat(scales, 16))        # 16-byte stride keeps scale pointers aligned
+    d_out = torch.full((total // 2,), 0xA5, dtype=torch.uint8, device="cuda")
+    d_os = torch.full((total // 32 * 16,), 0xA5, dtype=torch.uint8, device="cuda")
+    items, off = [], 0
+    host_scales = np.repeat(scales, 16)
+    for n in sizes:
+        b0 = off // 32
+        items.append((d_codes[off:off + n], d_scales[b0 * 16:b0 * 16 + n // 32], n, d_out[off // 2:(off + n) // 2],
+                      d_os[b0 * 16:b0 * 16 + n // 32]))
+        off += n
+    mxq.slice_scale_batched(items, "int8", "int4")
+    torch.cuda.synchronize()
+    got_c, got_s = to_host(d_out), to_host(d_os)
+    off = 0
+    for n in sizes:
+        b0 = off // 32
+        sc = host_scales[b0 * 16:b0 * 16 + n // 32]
+        wc, ws = orc.slice_scale(codes[off:off + n], sc, "int8", "int4")
+        assert bits_equal(got_c[off // 2:(off + n) // 2], orc.pack(wc, 4)), (count, off)
+        assert bits_equal(got_s[b0 * 16:b0 * 16 + n // 32], ws), (count, off)
+        assert np.all(got_s[b0 * 16 + n // 32:b0 * 16 + 16] == 0xA5) or n // 32 >= 16
+        off += n
+
+
 # ---------------------------------------------------------------------------------------------
 # Reconstruction
 # ---------------------------------------------------------------------------------------------
