@@ -63,7 +63,10 @@ STEP_BYTES_PER_ELEM = sum(OP_BYTES.values())
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (same workload, same launch configuration).  Valid only for the kernel sources the
 # capture was taken from: when their digest differs the bench reports traffic = null.
-NCU_TRAFFIC = {"fake_quant_bf16_via_anchor": 216_250_000}     # profiles/fake_quant_kernel_bf16_8192x8192_full.md
+NCU_TRAFFIC = {
+    "fake_quant_bf16_via_anchor": 216_250_000,   # profiles/fake_quant_kernel_bf16_8192x8192_full.md
+    "fake_quant_bwd_bf16": 213_500_000,          # profiles/bench_step_dram_counters_bf16_8192x8192.md
+}
 NCU_TRAFFIC_SOURCES = "421a29f0192ae1a6"
 
 
