@@ -6,7 +6,7 @@
 A *step* is one pass of the whole hot path over one tensor of the headline workload (a
 BF16 8192 x 8192 weight matrix, Student-t with outliers): quantize to the MXFP8 (E4M3) and
 MXINT8 anchors, Slice-and-Scale to MXFP6 (E2M3) / MXFP4 (E2M1) / MXINT6 / MXINT4, the same
-conversion through the batched entry point, reconstruction to BF16, the fused fake-quant
+conversion through the batched entry point, both MXFP targets from one read of the anchor, reconstruction to BF16, the fused fake-quant
 forward through the anchor and its straight-through backward.  Consumers read what the
 *previous* step produced (four buffer sets, each with its own copy of the input), so no kernel finds its input in L2.
 
@@ -52,6 +52,7 @@ OP_BYTES = {
     "ss_int8_int6": code_b(8) + SCALE_B + code_b(6) + SCALE_B,
     "ss_int8_int4": code_b(8) + SCALE_B + code_b(4) + SCALE_B,
     "ss_batched_e4m3_e2m1": code_b(8) + SCALE_B + code_b(4) + SCALE_B,
+    "ss_multi_e4m3_e2m3_e2m1": code_b(8) + SCALE_B + code_b(6) + SCALE_B + code_b(4) + SCALE_B,
     "dequantize_e2m1_bf16": code_b(4) + SCALE_B + 2,
     "dequantize_int4_bf16": code_b(4) + SCALE_B + 2,
     "fake_quant_bf16_via_anchor": 4.0,
@@ -176,7 +177,7 @@ class HotPath:
         for _ in range(self.NSETS):
             s = {}
             for name, bits in (("e4m3", 8), ("int8", 8), ("e2m3", 6), ("e2m1", 4), ("int6", 6), ("int4", 4),
-                               ("e2m1_b", 4)):
+                               ("e2m1_b", 4), ("e2m3_m", 6), ("e2m1_m", 4)):
                 s[name] = (torch.empty(n * bits // 8, **u8), torch.empty(nb, **u8))
             s["deq_e2m1"] = torch.empty(n, dtype=torch.bfloat16, device=device)
             s["deq_int4"] = torch.empty(n, dtype=torch.bfloat16, device=device)
@@ -212,6 +213,8 @@ class HotPath:
             lambda: mxq.slice_scale(*prev["int8"], n, "int8", "int6", BLOCK, *cur["int6"]),
             lambda: mxq.slice_scale(*prev["int8"], n, "int8", "int4", BLOCK, *cur["int4"]),
             lambda: mxq.slice_scale_batched(self.items[j], "e4m3", "e2m1", BLOCK),
+            lambda: mxq.slice_scale_multi(*prev["e4m3"], n, "e4m3", ("e2m3", "e2m1"), BLOCK,
+                                          (cur["e2m3_m"], cur["e2m1_m"])),
             lambda: mxq.dequantize(*prev["e2m1"], n, "e2m1", BLOCK, dst=cur["deq_e2m1"]),
             lambda: mxq.dequantize(*prev["int4"], n, "int4", BLOCK, dst=cur["deq_int4"]),
             lambda: mxq.fake_quant(x, "e2m3", BLOCK, mxq.FQ_VIA_ANCHOR, dst=cur["fq"]),
@@ -410,6 +413,8 @@ def oracle_step(x_bits: np.ndarray):
     c4, s4 = orc.slice_scale(ca, sa, "e4m3", "e2m1", BLOCK)
     orc.slice_scale(ci, si, "int8", "int6", BLOCK)
     c4i, s4i = orc.slice_scale(ci, si, "int8", "int4", BLOCK)
+    orc.slice_scale(ca, sa, "e4m3", "e2m1", BLOCK)
+    orc.slice_scale(ca, sa, "e4m3", "e2m3", BLOCK)           # the two-target conversion: both targets again
     orc.slice_scale(ca, sa, "e4m3", "e2m1", BLOCK)
     orc.dequantize(c4, s4, "e2m1", BLOCK, orc.BF16)
     orc.dequantize(c4i, s4i, "int4", BLOCK, orc.BF16)

@@ -117,6 +117,22 @@ int mxq_slice_scale(const void *codes, const uint8_t *scales, size_t n, int bloc
                     mxq_stream stream);
 
 /*
+ * Q_{h->l} for several targets at once (Sec. 3.5, Inference: one stored anchor, lower precisions
+ * on demand): the same results as `ntargets` calls of mxq_slice_scale with the same source.
+ * Consecutive targets (dst_fmts[0] with [1], [2] with [3]) that form one of the fused pairs --
+ * MXINT8 -> {MXINT6, MXINT4}, MXFP8 E4M3 -> {E2M3, E2M1}, {E3M2, E2M1}, {E3M2, E2M3}, in either order
+ * -- are produced by ONE pass over the anchor; any other legal target is produced by a pass of its own.
+ *   dst_fmts, out_codes, out_scales  [in] HOST arrays of `ntargets` entries (0 <= ntargets <=
+ *                                    MXQ_MULTI_TARGETS_MAX); the pointers inside are device pointers
+ *                                    with the requirements of mxq_slice_scale; outputs must not
+ *                                    overlap the inputs or one another
+ */
+#define MXQ_MULTI_TARGETS_MAX 8
+int mxq_slice_scale_multi(const void *codes, const uint8_t *scales, size_t n, int block, int src_fmt,
+                          int ntargets, const int *dst_fmts, void *const *out_codes,
+                          uint8_t *const *out_scales, mxq_stream stream);
+
+/*
  * Reconstruction V^_i = X P_i (Sec. 3.3, Notation) into FP32 or BF16, one
  * round-to-nearest-even rounding into the output type (exact unless the result falls
  * below the type's normal range; beyond its range it becomes +-Inf).  MXINT zero

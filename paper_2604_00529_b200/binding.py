@@ -65,6 +65,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_quantize.argtypes = [vp, i, sz, i, i, vp, vp, vp]
     L.mxq_slice_scale.argtypes = [vp, vp, sz, i, i, i, vp, vp, vp]
     L.mxq_dequantize.argtypes = [vp, vp, sz, i, i, vp, i, vp]
+    L.mxq_slice_scale_multi.argtypes = [vp, vp, sz, i, i, i, ctypes.POINTER(i), ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
+    L.mxq_slice_scale_multi.restype = i
     L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
@@ -147,6 +149,22 @@ def slice_scale(codes: torch.Tensor, scales: torch.Tensor, n: int, src_fmt: str,
                              FORMATS[dst_fmt], _dev(out_codes, "out_codes"), _dev(out_scales, "out_scales"),
                              _stream(stream)), "mxq_slice_scale")
     return out_codes, out_scales
+
+
+def slice_scale_multi(codes: torch.Tensor, scales: torch.Tensor, n: int, src_fmt: str, dst_fmts: Sequence[str],
+                      block: int = 32, outs: Optional[Sequence[Tuple[torch.Tensor, torch.Tensor]]] = None, stream=None):
+    """mxq_slice_scale_multi: one anchor -> several lower formats; returns [(codes, scales), ...]."""
+    L = load_library()
+    k = len(dst_fmts)
+    if outs is None:
+        outs = [(torch.empty(codes_bytes(n, f), dtype=torch.uint8, device=codes.device),
+                 torch.empty(n // block if block > 0 else 0, dtype=torch.uint8, device=codes.device)) for f in dst_fmts]
+    fm = (ctypes.c_int * k)(*[FORMATS[f] for f in dst_fmts])
+    oc = (ctypes.c_void_p * k)(*[_dev(c, "out_codes") for c, _ in outs])
+    os_ = (ctypes.c_void_p * k)(*[_dev(s, "out_scales") for _, s in outs])
+    _check(L.mxq_slice_scale_multi(_dev(codes, "codes"), _dev(scales, "scales"), n, block, FORMATS[src_fmt], k, fm, oc,
+                                   os_, _stream(stream)), "mxq_slice_scale_multi")
+    return list(outs)
 
 
 def dequantize(codes: torch.Tensor, scales: torch.Tensor, n: int, fmt: str, block: int = 32,

@@ -102,6 +102,42 @@ int mxq_slice_scale(const void* codes, const uint8_t* scales, size_t n, int bloc
                               static_cast<cudaStream_t>(stream));
 }
 
+int mxq_slice_scale_multi(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int ntargets,
+                          const int* dst_fmts, void* const* out_codes, uint8_t* const* out_scales, mxq_stream stream)
+{
+    if (ntargets < 0 || ntargets > MXQ_MULTI_TARGETS_MAX) return MXQ_ERR_SIZE;
+    if (ntargets == 0) return MXQ_OK;
+    if (!dst_fmts || !out_codes || !out_scales) return MXQ_ERR_NULL;
+    if (!valid_format(src_fmt)) return MXQ_ERR_FORMAT;
+    for (int t = 0; t < ntargets; ++t)
+        if (!valid_format(dst_fmts[t])) return MXQ_ERR_FORMAT;
+    if (int rc = check_sizes(n, block)) return rc;
+    if (n % 32) return MXQ_ERR_SIZE;
+    for (int t = 0; t < ntargets; ++t)
+        if (!ss_pair_ok(src_fmt, dst_fmts[t])) return MXQ_ERR_PAIR;
+    if (n == 0) return MXQ_OK;
+    if (!codes || !scales) return MXQ_ERR_NULL;
+    if (!aligned(codes, 32) || !aligned(scales, 16)) return MXQ_ERR_ALIGN;
+    for (int t = 0; t < ntargets; ++t) {
+        if (!out_codes[t] || !out_scales[t]) return MXQ_ERR_NULL;
+        if (!aligned(out_codes[t], 32) || !aligned(out_scales[t], 16)) return MXQ_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int t = 0;
+    while (t < ntargets) {
+        if (t + 1 < ntargets) {
+            const int rc = launch_slice_scale2(codes, scales, n, block, src_fmt, dst_fmts[t], dst_fmts[t + 1], out_codes[t],
+                                               out_scales[t], out_codes[t + 1], out_scales[t + 1], s);
+            if (rc == MXQ_OK) { t += 2; continue; }
+            if (rc != MXQ_ERR_PAIR) return rc;          // no fused kernel for this pair: one at a time
+        }
+        if (int rc = launch_slice_scale(codes, scales, n, block, src_fmt, dst_fmts[t], out_codes[t], out_scales[t], s))
+            return rc;
+        ++t;
+    }
+    return MXQ_OK;
+}
+
 int mxq_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dst_dtype,
                    mxq_stream stream)
 {

@@ -25,6 +25,11 @@ int launch_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, 
                       cudaStream_t stream);
 int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt,
                        void* out_codes, uint8_t* out_scales, cudaStream_t stream);
+// Anchor -> two lower formats in one pass.  Returns MXQ_ERR_PAIR when this pair of targets has no
+// fused instantiation (the caller then falls back to two single-target launches).
+int launch_slice_scale2(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt1,
+                        int dst_fmt2, void* out_codes1, uint8_t* out_scales1, void* out_codes2, uint8_t* out_scales2,
+                        cudaStream_t stream);
 int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
                       cudaStream_t stream);
 int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);

@@ -63,6 +63,18 @@ def test_argument_checks_answer_on_the_host(L):
     assert ss(A, A, 64, 32, F["int8"], F["int4"], None, A, None) == E_NULL
     assert ss(A, A, 64, 32, F["int8"], F["int4"], A + 4, A, None) == E_ALIGN
     assert ss(A, A, 48, 16, F["int8"], F["int4"], A, A, None) == E_SIZE      # code units are 32 wide
+    multi = L.mxq_slice_scale_multi
+    import ctypes as C
+    two = (C.c_int * 2)(F["int6"], F["int4"])
+    bad = (C.c_int * 2)(F["int6"], F["e2m1"])
+    ptrs = (C.c_void_p * 2)(A, A)
+    nul = (C.c_void_p * 2)(A, None)
+    assert multi(A, A, 64, 32, F["int8"], 2, bad, ptrs, ptrs, None) == E_PAIR
+    assert multi(A, A, 64, 32, F["int8"], 2, two, nul, ptrs, None) == E_NULL
+    assert multi(A, A, 64, 32, F["int8"], 9, two, ptrs, ptrs, None) == E_SIZE
+    assert multi(A, A, 64, 32, F["int8"], 0, None, None, None, None) == OK
+    assert multi(A, A, 65, 32, F["int8"], 2, two, ptrs, ptrs, None) == E_SIZE
+    assert multi(A, A, 64, 32, F["int8"], 2, None, ptrs, ptrs, None) == E_NULL
     dq = L.mxq_dequantize
     assert dq(A, A, 64, F["int4"], 32, A, 5, None) == E_FORMAT
     assert dq(A, None, 64, F["int4"], 32, A, 0, None) == E_NULL

@@ -10,7 +10,7 @@ import paper_2604_00529_b200 as mxq
 from oracle import mxq_oracle as orc
 from paper_2604_00529_b200 import inputs
 
-from gpu_util import (ALL_FORMATS, FP_FORMATS, INT_FORMATS, MAIN_FORMATS, bits_equal, first_diff, gpu_dequantize,
+from gpu_util import (ALL_FORMATS, FP_FORMATS, INT_FORMATS, MAIN_FORMATS, Guarded, bits_equal, first_diff, gpu_dequantize,
                       gpu_fake_quant, gpu_quantize, gpu_slice_scale, ss_pairs, to_dev, to_host)
 
 pytestmark = pytest.mark.gpu
@@ -215,6 +215,31 @@ def test_slice_scale_batched_item_counts(count):
         assert bits_equal(got_s[b0 * 16:b0 * 16 + n // 32], ws), (count, off)
         assert np.all(got_s[b0 * 16 + n // 32:b0 * 16 + 16] == 0xA5) or n // 32 >= 16
         off += n
+
+
+@pytest.mark.parametrize("src,dsts", [
+    ("int8", ["int6", "int4"]), ("int8", ["int4", "int6"]), ("e4m3", ["e2m3", "e2m1"]), ("e4m3", ["e2m1", "e3m2"]),
+    ("e4m3", ["e3m2", "e2m3"]), ("e4m3", ["e2m3", "e2m1", "e3m2"]), ("int8", ["int7", "int2"]), ("int8", ["int4"]),
+    ("e4m3", ["e3m2", "e2m3", "e2m1", "e2m2", "e3m3"]), ("int6", ["int4", "int3"]),
+], ids=lambda v: v if isinstance(v, str) else "+".join(v))
+@pytest.mark.parametrize("block", [32, 16, 128])
+def test_slice_scale_multi_equals_single_target_conversions(src, dsts, block):
+    """One read of the anchor, several targets: fused pairs in both orders, lists that mix fused and
+    single passes, and pairs that have no fused kernel."""
+    codes, scales32 = _all_codes_input(src, nblk_extra=301 * 4 - 256)
+    n = codes.size - codes.size % 128
+    codes = codes[:n]
+    scales = np.resize(scales32, n // block)
+    packed = orc.pack(codes, orc.bits(src))
+    guards = [(Guarded(mxq.codes_bytes(n, d)), Guarded(n // block)) for d in dsts]
+    mxq.slice_scale_multi(to_dev(packed), to_dev(scales), n, src, dsts, block, [(c.view, s.view) for c, s in guards])
+    torch.cuda.synchronize()
+    for d, (gc, gs) in zip(dsts, guards):
+        gc.check()
+        gs.check()
+        wc, ws = orc.slice_scale(codes, scales, src, d, block)
+        assert bits_equal(to_host(gs.view), ws), (d, first_diff(to_host(gs.view), ws))
+        assert bits_equal(to_host(gc.view), orc.pack(wc, orc.bits(d))), d
 
 
 # ---------------------------------------------------------------------------------------------
