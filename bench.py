@@ -65,10 +65,10 @@ STEP_BYTES_PER_ELEM = sum(OP_BYTES.values())
 # profiles/ (same workload, same launch configuration).  Valid only for the kernel sources the
 # capture was taken from: when their digest differs the bench reports traffic = null.
 NCU_TRAFFIC = {
-    "fake_quant_bf16_via_anchor": 216_250_000,   # profiles/fake_quant_kernel_bf16_8192x8192_full.md
-    "fake_quant_bwd_bf16": 213_500_000,          # profiles/bench_step_dram_counters_bf16_8192x8192.md
-}
-NCU_TRAFFIC_SOURCES = "421a29f0192ae1a6"
+    "fake_quant_bf16_via_anchor": 218203776,
+    "fake_quant_bwd_bf16": 214693248,
+}   # profiles/fake_quant_and_copy_kernels_bf16_8192x8192_full.md
+NCU_TRAFFIC_SOURCES = "ee278bc1119ff6ae"
 
 
 def kernel_sources_digest() -> str:
