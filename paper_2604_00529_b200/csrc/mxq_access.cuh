@@ -78,6 +78,30 @@ __device__ __forceinline__ void load_words(uint32_t (&w)[NW], const void* p)
     }
 }
 
+// Load NB bytes (any count) from `p`, which is aligned to piece_align(NB), into the low bytes of
+// the word array; bytes beyond NB are zero.
+template <int NB, int NW>
+__device__ __forceinline__ void load_bytes(uint32_t (&w)[NW], const void* p)
+{
+    static_assert(NW * 4 >= NB, "not enough words");
+    if constexpr (NB % 4 == 0) {
+        load_words<NB / 4>(w, p);
+    } else {
+        constexpr int A = piece_align(NB);                     // 1 or 2
+        const char* c = static_cast<const char*>(p);
+#pragma unroll
+        for (int i = 0; i < NW; ++i) w[i] = 0;
+        if constexpr (A == 2) {
+#pragma unroll
+            for (int i = 0; i < NB / 2; ++i)
+                w[i / 2] |= (uint32_t)*reinterpret_cast<const uint16_t*>(c + i * 2) << ((i & 1) * 16);
+        } else {
+#pragma unroll
+            for (int i = 0; i < NB; ++i) w[i / 4] |= (uint32_t)*reinterpret_cast<const uint8_t*>(c + i) << ((i & 3) * 8);
+        }
+    }
+}
+
 // Store the low NB bytes of the word array to `p`, which is aligned to piece_align(NB).
 template <int NB, int NW>
 __device__ __forceinline__ void store_bytes(void* p, const uint32_t (&w)[NW])

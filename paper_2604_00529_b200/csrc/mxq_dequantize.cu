@@ -5,20 +5,33 @@
 namespace mxq {
 namespace {
 
-constexpr int kU = 1;
+constexpr int kU = 2;
 constexpr int kThreads = 128;
 
 template <class F, class T>
 int run(const void* codes, const uint8_t* scales, size_t n, int block, void* dst, cudaStream_t stream)
 {
-    auto kern = dequantize_kernel<F, T, kU, kThreads>;
-    const size_t nunits = n / 32;
-    const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
-    int shift = 0, per_unit = 1;
-    if (block == 16) per_unit = 2;
-    else while ((32 << shift) < block) ++shift;
-    return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream, static_cast<const uint8_t*>(codes),
-                         scales, nunits, shift, per_unit, static_cast<uint8_t*>(dst));
+    if constexpr (T::size == 4) {
+        // FP32 output: lane units of 32 output bytes
+        auto kern = dequantize_wide_kernel<F, T, kU, kThreads>;
+        const size_t nunits = n / T::epl;
+        const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
+        int shift = 0;
+        while ((T::epl << shift) < block) ++shift;        // units per scale = block / epl (block >= 16 >= epl)
+        return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream,
+                             static_cast<const uint8_t*>(codes), scales, nunits, shift, static_cast<uint8_t*>(dst));
+    } else {
+        // 16-bit output: lane units of 32 codes
+        auto kern = dequantize_kernel<F, T, kU, kThreads>;
+        const size_t nunits = n / 32;
+        const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
+        int shift = 0, per_unit = 1;
+        if (block == 16) per_unit = 2;
+        else while ((32 << shift) < block) ++shift;
+        return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream,
+                             static_cast<const uint8_t*>(codes), scales, nunits, shift, per_unit,
+                             static_cast<uint8_t*>(dst));
+    }
 }
 
 }  // namespace

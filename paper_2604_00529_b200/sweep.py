@@ -1,0 +1,181 @@
+"""Bandwidth sweep of libmxq on one GPU.
+
+    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--json out.json]
+
+For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
+for every anchor-to-lower pair, reconstruction and the fused fake-quant, timed with CUDA events over
+back-to-back launches that rotate over enough buffer copies to exceed the 126 MB L2 (small sizes
+therefore show launch-bound, not cache-resident, figures).  GB/s counts algorithmic bytes (read +
+written).  `--model` adds the whole-model conversion of an 8B Llama-shaped weight set (224 tensors,
+6.98 G elements) through one batched launch per target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+import paper_2604_00529_b200 as mxq
+from paper_2604_00529_b200 import inputs
+
+BLOCK = 32
+L2_BYTES = 126 << 20
+
+
+def _peak():
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def _time(launch, copies: int, reps: int) -> float:
+    """Average microseconds per launch; launch(j) must use buffer copy j."""
+    for j in range(min(3, copies)):
+        launch(j)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(reps):
+        launch(i % copies)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) * 1e3 / reps
+
+
+def sweep_size(n: int, base_dev: torch.Tensor, reps: int):
+    """All ops at n elements; returns {op: (us, GB/s)}."""
+    bits = {"int8": 8, "int6": 6, "int4": 4, "e4m3": 8, "e3m2": 6, "e2m3": 6, "e2m1": 4}
+    # enough rotating copies that a buffer is not found in L2 again (at least 2, at most 2048)
+    copies = int(min(2048, max(2, -(-2 * L2_BYTES // (2 * n)))))
+    if n * 2 * copies > 24 << 30:
+        copies = 2
+    xs = [base_dev[:n].clone() if n <= base_dev.numel() else base_dev.repeat(n // base_dev.numel()) for _ in range(copies)]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    out = {}
+
+    def rec(name, us, bytes_per_elem):
+        out[name] = (us, bytes_per_elem * n / us / 1e3)
+
+    anchors = {}
+    for fmt in ("int8", "e4m3", "int6", "int4", "e2m3", "e2m1"):
+        cs = [(torch.empty(n * bits[fmt] // 8, **u8), torch.empty(n // BLOCK, **u8)) for _ in range(copies)]
+        us = _time(lambda j: mxq.quantize(xs[j], fmt, BLOCK, *cs[j]), copies, reps)
+        rec("quantize_bf16_" + fmt, us, 2 + bits[fmt] / 8 + 1 / BLOCK)
+        if fmt in ("int8", "e4m3"):
+            anchors[fmt] = cs
+        else:
+            del cs
+    for src, dsts in (("int8", ("int6", "int4")), ("e4m3", ("e2m3", "e3m2", "e2m1"))):
+        for dst in dsts:
+            os_ = [(torch.empty(n * bits[dst] // 8, **u8), torch.empty(n // BLOCK, **u8)) for _ in range(copies)]
+            us = _time(lambda j: mxq.slice_scale(*anchors[src][j], n, src, dst, BLOCK, *os_[j]), copies, reps)
+            rec("slice_scale_%s_%s" % (src, dst), us, 1 + bits[dst] / 8 + 2 / BLOCK)
+            if dst in ("int4", "e2m1"):
+                ys = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+                us = _time(lambda j: mxq.dequantize(*os_[j], n, dst, BLOCK, dst=ys[j]), copies, reps)
+                rec("dequantize_%s_bf16" % dst, us, bits[dst] / 8 + 1 / BLOCK + 2)
+                del ys
+            del os_
+    two = [[(torch.empty(n * 6 // 8, **u8), torch.empty(n // BLOCK, **u8)), (torch.empty(n // 2, **u8), torch.empty(n // BLOCK, **u8))]
+           for _ in range(copies)]
+    us = _time(lambda j: mxq.slice_scale_multi(*anchors["e4m3"][j], n, "e4m3", ("e2m3", "e2m1"), BLOCK, two[j]), copies, reps)
+    rec("slice_scale_multi_e4m3_e2m3+e2m1", us, 1 + 6 / 8 + 4 / 8 + 3 / BLOCK)
+    del two, anchors
+    ys = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+    for fmt, mode, tag in (("e2m3", mxq.FQ_VIA_ANCHOR, "via_anchor"), ("int4", mxq.FQ_DIRECT, "direct")):
+        us = _time(lambda j: mxq.fake_quant(xs[j], fmt, BLOCK, mode, dst=ys[j]), copies, reps)
+        rec("fake_quant_bf16_%s_%s" % (fmt, tag), us, 4.0)
+    return out, copies
+
+
+def sweep_f32(n: int, reps: int):
+    """The FP32 entry points at one size (workload 1's element type)."""
+    x = torch.from_numpy(inputs.weight_f32_normal(n // 4096, 4096, seed=0)).cuda()
+    copies = 6
+    xs = [x.clone() for _ in range(copies)]
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    cs = [(torch.empty(n, **u8), torch.empty(n // BLOCK, **u8)) for _ in range(copies)]
+    ys = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(copies)]
+    out = {}
+    for fmt in ("int8", "e4m3"):
+        us = _time(lambda j: mxq.quantize(xs[j], fmt, BLOCK, *cs[j]), copies, reps)
+        out["quantize_f32_" + fmt] = (us, (4 + 1 + 1 / BLOCK) * n / us / 1e3)
+        us = _time(lambda j: mxq.dequantize(*cs[j], n, fmt, BLOCK, dst=ys[j]), copies, reps)
+        out["dequantize_%s_f32" % fmt] = (us, (1 + 1 / BLOCK + 4) * n / us / 1e3)
+        us = _time(lambda j: mxq.fake_quant(xs[j], fmt, BLOCK, mxq.FQ_DIRECT, dst=ys[j]), copies, reps)
+        out["fake_quant_f32_" + fmt] = (us, 8.0 * n / us / 1e3)
+    return out
+
+
+def whole_model(reps: int = 5):
+    """Anchor -> target for the 224 tensors of the 8B Llama-shaped set, one batched launch per target.
+    Anchors hold seeded random codes (the conversion's speed does not depend on the values)."""
+    shapes = inputs.llama8b_shapes()
+    total = sum(r * c for *_, r, c in shapes)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    out = {}
+    for anchor, dsts in (("int8", (("int6", 6), ("int4", 4))), ("e4m3", (("e2m3", 6), ("e2m1", 4)))):
+        codes = torch.randint(0, 127, (total,), dtype=torch.uint8, device="cuda", generator=g)   # no E4M3 NaN codes
+        scales = torch.randint(100, 140, (total // BLOCK,), dtype=torch.uint8, device="cuda", generator=g)
+        for dst, b in dsts:
+            oc = torch.empty(total * b // 8, dtype=torch.uint8, device="cuda")
+            os_ = torch.empty(total // BLOCK, dtype=torch.uint8, device="cuda")
+            items, off = [], 0
+            for *_, r, c in shapes:
+                n = r * c
+                items.append((codes[off:off + n], scales[off // BLOCK:(off + n) // BLOCK], n,
+                              oc[off * b // 8:(off + n) * b // 8], os_[off // BLOCK:(off + n) // BLOCK]))
+                off += n
+            table = mxq.make_items(items)
+            us = _time(lambda j: mxq.slice_scale_batched(table, anchor, dst, BLOCK), 1, reps)
+            per = _time(lambda j: [mxq.slice_scale(c_, s_, n_, anchor, dst, BLOCK, oc_, os2) for c_, s_, n_, oc_, os2 in items], 1, reps)
+            bytes_ = total * (1 + b / 8 + 2 / BLOCK)
+            out["model_%s_%s" % (anchor, dst)] = {"batched_ms": us / 1e3, "batched_gbs": bytes_ / us / 1e3,
+                                                  "per_tensor_launches_ms": per / 1e3, "per_tensor_gbs": bytes_ / per / 1e3,
+                                                  "elements": total, "tensors": len(items)}
+            del oc, os_, table, items
+        del codes, scales
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--min-log2", type=int, default=16)
+    ap.add_argument("--max-log2", type=int, default=31)
+    ap.add_argument("--model", action="store_true")
+    ap.add_argument("--json", default=None)
+    args = ap.parse_args()
+    mxq.load_library()
+    peak, kind = _peak()
+    base = torch.from_numpy(inputs.flat_bf16_normal(1 << 27, seed=5).view(np.int16)).cuda().view(torch.bfloat16)
+    result = {"peak_gbs": peak, "peak_kind": kind, "sizes": {}, "f32": {}, "model": {}}
+    for k in range(args.min_log2, args.max_log2 + 1):
+        n = 1 << k
+        reps = 200 if k <= 22 else (50 if k <= 27 else 10)
+        ops, copies = sweep_size(n, base, reps)
+        result["sizes"][k] = {name: {"us": round(us, 3), "gbs": round(g, 1)} for name, (us, g) in ops.items()}
+        print("2^%d elements (%d buffer copies)" % (k, copies))
+        for name, (us, g) in ops.items():
+            print("  %-36s %10.2f us %8.1f GB/s  %5.1f %% of %s peak  %5.1f %% of 8000" % (name, us, g, 100 * g / peak, kind, g / 80))
+        torch.cuda.empty_cache()
+    f32 = sweep_f32(1 << 26, 50)
+    result["f32"] = {name: {"us": round(us, 3), "gbs": round(g, 1)} for name, (us, g) in f32.items()}
+    print("FP32 entry points, 2^26 elements")
+    for name, (us, g) in f32.items():
+        print("  %-36s %10.2f us %8.1f GB/s  %5.1f %% of %s peak" % (name, us, g, 100 * g / peak, kind))
+    if args.model:
+        result["model"] = whole_model()
+        for name, r in result["model"].items():
+            print("  %-20s batched %.3f ms %7.1f GB/s | %d separate launches %.3f ms %7.1f GB/s" %
+                  (name, r["batched_ms"], r["batched_gbs"], r["tensors"], r["per_tensor_launches_ms"], r["per_tensor_gbs"]))
+    if args.json:
+        json.dump(result, open(args.json, "w"), indent=1)
+
+
+if __name__ == "__main__":
+    main()
