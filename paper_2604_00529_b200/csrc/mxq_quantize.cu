@@ -6,9 +6,7 @@
 namespace mxq {
 namespace {
 
-// lane units in flight per thread: the MXINT quantizer is bound by its integer arithmetic and gains
-// from more independent work per thread; the MXFP one is bound by HBM alone
-template <class F> constexpr int kU = F::kind == KIND_INT ? 4 : 2;
+constexpr int kU = 2;   // lane units in flight per thread
 constexpr int kThreads = 128;
 
 template <class T, class F, int BLOCK>
@@ -17,7 +15,7 @@ int run(const void* src, size_t n, void* codes, uint8_t* scales, cudaStream_t st
     if constexpr (BLOCK < T::epl) {
         return MXQ_ERR_BLOCK;
     } else {
-        constexpr int U = kU<F>;
+        constexpr int U = kU;
         auto kern = quantize_kernel<T, F, BLOCK, U, kThreads>;
         const size_t nunits = n / T::epl;
         const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
