@@ -143,6 +143,21 @@ int mxq_dequantize(const void *codes, const uint8_t *scales, size_t n, int fmt, 
                    void *dst, int dst_dtype, mxq_stream stream);
 
 /*
+ * Scales for the matrix multiply that consumes the converted weights (Sec. 3.5: W_t feeds the
+ * layer's matmul).  Blackwell's block-scaled tensor-core multiply reads the E8M0 bytes of a
+ * [rows, kblocks] scale matrix (kblocks = columns / 32, row-major as every entry point above
+ * writes them) in tiles of 128 rows x 4 block-columns: a tile is 512 consecutive bytes, the byte
+ * of row r and column c inside it sits at (r mod 32) * 16 + (r div 32) * 4 + c, and tiles follow
+ * one another row-tile by row-tile.  mxq_tile_scales writes that order; rows and columns beyond
+ * the matrix are filled with byte 0.  The element codes need no rearrangement: FP8 codes are
+ * bytes, FP6 / FP4 codes are already the packed little-endian streams the hardware unpacks.
+ *   scales [in]  device, rows * kblocks bytes, 16-byte aligned
+ *   tiled  [out] device, mxq_tiled_scales_bytes(rows, kblocks) bytes, 16-byte aligned, no overlap
+ */
+size_t mxq_tiled_scales_bytes(size_t rows, size_t kblocks);
+int mxq_tile_scales(const uint8_t *scales, size_t rows, size_t kblocks, uint8_t *tiled, mxq_stream stream);
+
+/*
  * Fused fake-quant forward, Eq. 6 in reconstructed form; nothing but the result leaves
  * the SM.  mode MXQ_FQ_DIRECT: dst = dequantize(Q_fmt(src)).  mode MXQ_FQ_VIA_ANCHOR:
  * dst = dequantize(Q_{A->fmt}(Q_A(src))) with A = MXINT8 for MXINT targets and MXFP8 E4M3

@@ -384,6 +384,27 @@ int mxo_fake_quant_bwd(const void *grad_out, int dtype, size_t n, void *grad_in)
 }
 
 /* ------------------------------------------------------------------------- */
+/* Scale bytes in the tiled order of a block-scaled matrix multiply           */
+/* ------------------------------------------------------------------------- */
+
+/* [rows, kblocks] row-major -> tiles of 128 rows x 4 columns, 512 bytes each, tiles ordered
+ * row-tile by row-tile; inside a tile the byte of (r, c) sits at (r mod 32)*16 + (r div 32)*4 + c.
+ * Bytes that no (r, c) of the matrix maps to are 0.  `out` holds
+ * ceil(rows/128) * ceil(kblocks/4) * 512 bytes. */
+int mxo_tile_scales(const uint8_t *scales, size_t rows, size_t kblocks, uint8_t *out)
+{
+    size_t col_tiles = (kblocks + 3) / 4, row_tiles = (rows + 127) / 128;
+    memset(out, 0, row_tiles * col_tiles * 512);
+    for (size_t r = 0; r < rows; ++r)
+        for (size_t c = 0; c < kblocks; ++c) {
+            size_t tile = (r / 128) * col_tiles + c / 4;
+            size_t rr = r % 128, cc = c % 4;
+            out[tile * 512 + (rr % 32) * 16 + (rr / 32) * 4 + cc] = scales[r * kblocks + c];
+        }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Packed storage: little-endian bitstream, element i at bits [i*bits,(i+1)*bits) */
 /* ------------------------------------------------------------------------- */
 

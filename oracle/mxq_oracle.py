@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
             L.mxo_fake_quant.argtypes = [c_vp, c_int, c_sz, c_int, c_int, c_int, c_int, c_int, c_vp]
             L.mxo_fake_quant_bwd.argtypes = [c_vp, c_int, c_sz, c_vp]
             L.mxo_pack.argtypes = [c_vp, c_sz, c_int, c_vp]
+            L.mxo_tile_scales.argtypes = [c_vp, c_sz, c_sz, c_vp]
             L.mxo_unpack.argtypes = [c_vp, c_sz, c_int, c_vp]
             _lib = L
     return _lib
@@ -189,6 +190,15 @@ def fake_quant_bwd(g: np.ndarray) -> np.ndarray:
     g, dt = _src(g)
     out = np.empty_like(g)
     lib().mxo_fake_quant_bwd(_ptr(g), dt, g.size, _ptr(out))
+    return out
+
+
+def tile_scales(scales: np.ndarray, rows: int, kblocks: int) -> np.ndarray:
+    """Row-major [rows, kblocks] scale bytes in the 128 x 4 tiled order of a block-scaled matmul."""
+    scales = np.ascontiguousarray(scales, np.uint8)
+    assert scales.size == rows * kblocks
+    out = np.empty(-(-rows // 128) * -(-kblocks // 4) * 512, np.uint8)
+    lib().mxo_tile_scales(_ptr(scales), rows, kblocks, _ptr(out))
     return out
 
 

@@ -68,6 +68,10 @@ def load_library() -> ctypes.CDLL:
     L.mxq_slice_scale_multi.argtypes = [vp, vp, sz, i, i, i, ctypes.POINTER(i), ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
     L.mxq_slice_scale_multi.restype = i
     L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
+    L.mxq_tiled_scales_bytes.argtypes = [sz, sz]
+    L.mxq_tiled_scales_bytes.restype = sz
+    L.mxq_tile_scales.argtypes = [vp, sz, sz, vp, vp]
+    L.mxq_tile_scales.restype = i
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
     L.mxq_slice_scale_batched_static.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
@@ -176,6 +180,22 @@ def dequantize(codes: torch.Tensor, scales: torch.Tensor, n: int, fmt: str, bloc
     _check(L.mxq_dequantize(_dev(codes, "codes"), _dev(scales, "scales"), n, FORMATS[fmt], block, _dev(dst, "dst"),
                             _dtype_id(dst), _stream(stream)), "mxq_dequantize")
     return dst
+
+
+def tiled_scales_bytes(rows: int, kblocks: int) -> int:
+    return load_library().mxq_tiled_scales_bytes(rows, kblocks)
+
+
+def tile_scales(scales: torch.Tensor, rows: int, kblocks: int, tiled: Optional[torch.Tensor] = None,
+                stream=None) -> torch.Tensor:
+    """mxq_tile_scales: row-major [rows, kblocks] scale bytes -> the 128 x 4 tiled order a block-scaled
+    tensor-core matmul reads."""
+    L = load_library()
+    if tiled is None:
+        tiled = torch.empty(tiled_scales_bytes(rows, kblocks), dtype=torch.uint8, device=scales.device)
+    _check(L.mxq_tile_scales(_dev(scales, "scales"), rows, kblocks, _dev(tiled, "tiled"), _stream(stream)),
+           "mxq_tile_scales")
+    return tiled
 
 
 def fake_quant(src: torch.Tensor, fmt: str, block: int = 32, mode: int = FQ_DIRECT,

@@ -75,6 +75,12 @@ def test_argument_checks_answer_on_the_host(L):
     assert multi(A, A, 64, 32, F["int8"], 0, None, None, None, None) == OK
     assert multi(A, A, 65, 32, F["int8"], 2, two, ptrs, ptrs, None) == E_SIZE
     assert multi(A, A, 64, 32, F["int8"], 2, None, ptrs, ptrs, None) == E_NULL
+    ts = L.mxq_tile_scales
+    assert ts(None, 0, 4, None, None) == OK and ts(A, 128, 0, A, None) == OK
+    assert ts(None, 128, 4, A, None) == E_NULL and ts(A, 128, 4, None, None) == E_NULL
+    assert ts(A + 4, 128, 4, A, None) == E_ALIGN and ts(A, 128, 4, A + 8, None) == E_ALIGN
+    assert L.mxq_tiled_scales_bytes(1, 1) == 512 and L.mxq_tiled_scales_bytes(129, 5) == 2 * 2 * 512
+    assert L.mxq_tiled_scales_bytes(8192, 256) == 8192 * 256
     dq = L.mxq_dequantize
     assert dq(A, A, 64, F["int4"], 32, A, 5, None) == E_FORMAT
     assert dq(A, None, 64, F["int4"], 32, A, 0, None) == E_NULL

@@ -353,3 +353,43 @@ def test_smallest_and_empty_inputs():
     c, s = mxq.quantize(empty, "int8")
     assert c.numel() == 0 and s.numel() == 0
     assert mxq.fake_quant(empty, "e2m1").numel() == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# The tensor-level study of Sec. 4.3 / App. C through the CUDA path
+# ---------------------------------------------------------------------------------------------
+
+def test_tensor_level_mse_study_on_gpu():
+    """100 random tensors of shape (1, 1024): Slice-and-Scale against direct quantization over bit-widths
+    at block 64 and over block sizes at 4 bits.  The GPU's reconstruction errors must equal the
+    oracle's (the outputs are bit-identical) and show what the paper reports: SS tracks direct
+    quantization closely, the gap being largest for MXFP at intermediate widths."""
+    rng = np.random.default_rng(100)
+    x = rng.standard_normal(100 * 1024).astype(np.float32)
+
+    def mse(y):
+        return float(np.mean((y.astype(np.float64) - x) ** 2))
+
+    table = {}
+    for fmt in ("int2", "int3", "int4", "int5", "int6", "int7", "int8", "e2m1", "e2m2", "e3m2", "e2m3", "e3m3", "e4m3"):
+        for mode in (orc.FQ_DIRECT, orc.FQ_VIA_ANCHOR):
+            got = gpu_fake_quant(x, fmt, 64, mode)
+            want = orc.fake_quant(x, fmt, 64, mode)
+            assert bits_equal(got, want), (fmt, mode, first_diff(got, want))
+            table[(fmt, mode)] = mse(got)
+    for fmt in ("int2", "int3", "int4", "int5", "int6", "int7", "e2m1", "e2m2", "e3m2", "e3m3"):
+        r = table[(fmt, orc.FQ_VIA_ANCHOR)] / table[(fmt, orc.FQ_DIRECT)]
+        assert 1.0 <= r < 2.0, (fmt, r)
+    gap = {f: table[(f, orc.FQ_VIA_ANCHOR)] / table[(f, orc.FQ_DIRECT)] for f in ("e2m1", "e2m2", "e3m2", "e3m3")}
+    assert min(gap["e2m2"], gap["e3m2"]) > max(gap["e2m1"], gap["e3m3"])
+    for f in ("int8", "e4m3"):                                    # the anchor itself: both routes coincide
+        assert table[(f, orc.FQ_VIA_ANCHOR)] == table[(f, orc.FQ_DIRECT)]
+    by_block = []
+    for block in (16, 32, 64, 128):
+        d = gpu_fake_quant(x, "int4", block, orc.FQ_DIRECT)
+        s = gpu_fake_quant(x, "int4", block, orc.FQ_VIA_ANCHOR)
+        assert bits_equal(d, orc.fake_quant(x, "int4", block, orc.FQ_DIRECT))
+        assert bits_equal(s, orc.fake_quant(x, "int4", block, orc.FQ_VIA_ANCHOR))
+        by_block.append((mse(d), mse(s)))
+    assert all(a[0] < b[0] and a[1] < b[1] for a, b in zip(by_block[:-1], by_block[1:]))   # smaller blocks, lower error
+    assert all(1.0 <= s / d < 1.2 for d, s in by_block)

@@ -1,0 +1,103 @@
+"""The tiled scale order for block-scaled matrix multiplies: the oracle against a hand-worked case
+and a second formulation (CPU), the CUDA entry point against the oracle, and -- the pin that counts --
+a block-scaled tensor-core matmul of the library in use fed with our codes and tiled scales (GPU)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2604_00529_b200 as mxq
+from oracle import mxq_oracle as orc
+from paper_2604_00529_b200 import inputs
+
+
+def _by_reshapes(s: np.ndarray) -> np.ndarray:
+    """Second formulation: pad to whole tiles, split into (row tile, 128, column tile, 4), bring the two
+    tile indices to the front, then reorder each 128 x 4 tile as (4 groups of 32 rows) -> (32, 4, 4)."""
+    rows, kb = s.shape
+    rt, ct = -(-rows // 128), -(-kb // 4)
+    p = np.zeros((rt * 128, ct * 4), np.uint8)
+    p[:rows, :kb] = s
+    t = p.reshape(rt, 128, ct, 4).transpose(0, 2, 1, 3)            # [rt, ct, 128, 4]
+    t = t.reshape(rt * ct, 4, 32, 4).transpose(0, 2, 1, 3)          # [tile, 32, 4 groups, 4 cols]
+    return np.ascontiguousarray(t).reshape(-1)
+
+
+def test_oracle_tiled_order_hand_worked():
+    rows, kb = 33, 5
+    s = (np.arange(rows * kb) % 251 + 1).astype(np.uint8).reshape(rows, kb)
+    t = orc.tile_scales(s, rows, kb)
+    assert t.size == 1 * 2 * 512
+    assert t[0] == s[0, 0] and t[16] == s[1, 0] and t[4] == s[32, 0] and t[7] == s[32, 3]
+    assert t[31 * 16 + 1] == s[31, 1] and t[512] == s[0, 4] and t[512 + 16 * 5] == s[5, 4]
+    assert t[8] == 0 and t[512 + 1] == 0                             # rows 64.. and column 5 do not exist
+    assert np.count_nonzero(t) == rows * kb
+
+
+@pytest.mark.parametrize("rows,kb", [(1, 1), (128, 4), (129, 4), (128, 5), (300, 7), (4096, 128), (1000, 33)])
+def test_oracle_tiled_order_second_formulation(rows, kb):
+    s = np.random.default_rng(rows * 1000 + kb).integers(0, 256, (rows, kb)).astype(np.uint8)
+    assert np.array_equal(orc.tile_scales(s, rows, kb), _by_reshapes(s))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows,kb", [(1, 1), (128, 4), (129, 4), (128, 5), (300, 7), (4096, 128), (1000, 33), (8192, 256)])
+def test_gpu_tile_scales_matches_oracle(rows, kb):
+    s = np.random.default_rng(rows + kb).integers(0, 256, (rows, kb)).astype(np.uint8)
+    nbytes = mxq.tiled_scales_bytes(rows, kb)
+    buf = torch.full((nbytes + 512,), 0xA5, dtype=torch.uint8, device="cuda")
+    mxq.tile_scales(torch.from_numpy(s).cuda(), rows, kb, buf[256:256 + nbytes])
+    torch.cuda.synchronize()
+    got = buf.cpu().numpy()
+    assert np.array_equal(got[256:256 + nbytes], orc.tile_scales(s, rows, kb))
+    assert np.all(got[:256] == 0xA5) and np.all(got[256 + nbytes:] == 0xA5)
+
+
+def _mixed_matrix(rows, cols, seed):
+    """Rows and 32-wide blocks at very different magnitudes, so that a misplaced scale is a gross error."""
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((rows, cols))
+    x *= 2.0 ** rng.integers(-6, 7, (rows, 1))
+    x *= 2.0 ** rng.integers(-4, 5, (rows, cols // 32)).repeat(32, axis=1)
+    return inputs.to_bf16_bits(x.astype(np.float32).reshape(-1))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("fmt", ["e4m3", "e2m1"])
+def test_block_scaled_matmul_consumes_codes_and_tiled_scales(fmt):
+    """A = [M, K], B = [N, K] quantized along K with block 32; the library's block-scaled matmul on our
+    codes and tiled scales must equal dequantize(A) @ dequantize(B)^T."""
+    try:
+        from torch.nn.functional import ScalingType, SwizzleType, scaled_mm
+    except ImportError:
+        pytest.skip("this torch has no scaled_mm")
+    M, N, K = 256, 384, 1024
+    qa = {}
+    for name, rows, seed in (("a", M, 1), ("b", N, 2)):
+        bits = _mixed_matrix(rows, K, seed)
+        x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+        codes, scales = mxq.quantize(x, fmt, 32)
+        deq = mxq.dequantize(codes, scales, rows * K, fmt, 32, dtype=torch.float32).view(rows, K)
+        tiled = mxq.tile_scales(scales, rows, K // 32)
+        qa[name] = (codes, tiled, deq)
+    ref = qa["a"][2].double() @ qa["b"][2].double().t()
+    if fmt == "e4m3":
+        a = qa["a"][0].view(torch.float8_e4m3fn).view(M, K)
+        b = qa["b"][0].view(torch.float8_e4m3fn).view(N, K)
+    else:
+        a = qa["a"][0].view(torch.float4_e2m1fn_x2).view(M, K // 2)
+        b = qa["b"][0].view(torch.float4_e2m1fn_x2).view(N, K // 2)
+    sa = qa["a"][1].view(torch.float8_e8m0fnu)
+    sb = qa["b"][1].view(torch.float8_e8m0fnu)
+    try:
+        out = scaled_mm(a, b.t(), sa, ScalingType.BlockWise1x32, sb, ScalingType.BlockWise1x32,
+                        swizzle_a=SwizzleType.SWIZZLE_32_4_4, swizzle_b=SwizzleType.SWIZZLE_32_4_4,
+                        output_dtype=torch.bfloat16)
+    except (RuntimeError, NotImplementedError, ValueError) as e:
+        pytest.skip("block-scaled matmul not available for %s here: %s" % (fmt, str(e).splitlines()[0][:200]))
+    torch.cuda.synchronize()
+    err = (out.double() - ref).abs()
+    # BF16 output (8 significant bits) of an FP32 accumulation: a few 2^-8 relative to the row's scale
+    tol = 2.0 ** -6 * ref.abs().max(dim=1, keepdim=True).values + 1e-30
+    assert bool((err <= tol).all()), "max error / tolerance = %.3g" % float((err / tol).max())
+    # and the result is not trivially small: the check has teeth
+    assert float(ref.abs().max()) > 0
