@@ -168,6 +168,23 @@ int mxq_fake_quant(const void *src, int dtype, size_t n, int fmt, int block, int
                    void *dst, mxq_stream stream);
 
 /*
+ * mxq_fake_quant over `count` tensors in one launch (Sec. 3.5, Training: every quantized weight of
+ * the model goes through Eq. 6 in every step).  `items` is a HOST array, free to reuse when the call
+ * returns; every pointer inside is a device pointer with the requirements of mxq_fake_quant, and
+ * dst == src is allowed per item.  All tensors share dtype, format, block and mode.  The item table
+ * travels in the kernel's parameter space, 512 tensors per launch; more are split over several
+ * launches.  Nothing is allocated on the device.
+ */
+typedef struct {
+    const void *src;
+    void *dst;
+    size_t n;
+} mxq_fq_item;
+
+int mxq_fake_quant_batched(const mxq_fq_item *items, int count, int dtype, int fmt, int block, int mode,
+                           mxq_stream stream);
+
+/*
  * Straight-through estimator backward of mxq_fake_quant (Sec. 3.5): grad_in = grad_out.
  * grad_in == grad_out is a no-op; otherwise n elements of `dtype` are copied.
  */

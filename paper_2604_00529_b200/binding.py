@@ -30,6 +30,10 @@ class MxqError(RuntimeError):
         super().__init__("%s failed: %s" % (what, status_string(status)))
 
 
+class _FqItem(ctypes.Structure):
+    _fields_ = [("src", ctypes.c_void_p), ("dst", ctypes.c_void_p), ("n", ctypes.c_size_t)]
+
+
 class _Item(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("n", ctypes.c_size_t),
                 ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p)]
@@ -68,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_slice_scale_multi.argtypes = [vp, vp, sz, i, i, i, ctypes.POINTER(i), ctypes.POINTER(vp), ctypes.POINTER(vp), vp]
     L.mxq_slice_scale_multi.restype = i
     L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
+    L.mxq_fake_quant_batched.argtypes = [ctypes.POINTER(_FqItem), i, i, i, i, i, vp]
+    L.mxq_fake_quant_batched.restype = i
     L.mxq_tiled_scales_bytes.argtypes = [sz, sz]
     L.mxq_tiled_scales_bytes.restype = sz
     L.mxq_tile_scales.argtypes = [vp, sz, sz, vp, vp]
@@ -207,6 +213,38 @@ def fake_quant(src: torch.Tensor, fmt: str, block: int = 32, mode: int = FQ_DIRE
     _check(L.mxq_fake_quant(_dev(src, "src"), _dtype_id(src), src.numel(), FORMATS[fmt], block, mode,
                             _dev(dst, "dst"), _stream(stream)), "mxq_fake_quant")
     return dst
+
+
+class FqTable:
+    """A marshalled mxq_fq_item array for tensors that persist (e.g. a model's weights): build it once
+    with ``make_fq_items`` and pass it to ``fake_quant_batched`` every step."""
+
+    def __init__(self, pairs):
+        self.tensors = [(s, d if d is not None else s) for s, d in pairs]
+        if not self.tensors:
+            raise ValueError("no tensors")
+        self.dtype = _dtype_id(self.tensors[0][0])
+        self.array = (_FqItem * len(self.tensors))()
+        for k, (s, d) in enumerate(self.tensors):
+            if _dtype_id(s) != self.dtype or d.dtype != s.dtype or d.numel() != s.numel():
+                raise TypeError("all tensors of a batch share one dtype; dst matches src")
+            self.array[k] = _FqItem(_dev(s, "src"), _dev(d, "dst"), s.numel())
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_fq_items(pairs) -> FqTable:
+    """Marshal (src, dst) tensor pairs (dst None = in place) into an mxq_fq_item array."""
+    return FqTable(pairs)
+
+
+def fake_quant_batched(pairs, fmt: str, block: int = 32, mode: int = FQ_DIRECT, stream=None) -> None:
+    """mxq_fake_quant_batched over (src, dst) pairs or an FqTable made from them."""
+    L = load_library()
+    table = pairs if isinstance(pairs, FqTable) else FqTable(pairs)
+    _check(L.mxq_fake_quant_batched(table.array, len(table), table.dtype, FORMATS[fmt], block, mode, _stream(stream)),
+           "mxq_fake_quant_batched")
 
 
 def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

@@ -161,6 +161,51 @@ int mxq_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, int
     return launch_fake_quant(src, dtype, n, fmt, block, mode, dst, static_cast<cudaStream_t>(stream));
 }
 
+int mxq_fake_quant_batched(const mxq_fq_item* items, int count, int dtype, int fmt, int block, int mode,
+                           mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(dtype)) return MXQ_ERR_FORMAT;
+    if (mode != MXQ_FQ_DIRECT && mode != MXQ_FQ_VIA_ANCHOR) return MXQ_ERR_FORMAT;
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+    const size_t epl = dtype == MXQ_F32 ? 8 : 16;           // elements per 32-byte lane unit
+    for (int i = 0; i < count; ++i) {
+        const mxq_fq_item& it = items[i];
+        if (it.n % (size_t)block) return MXQ_ERR_SIZE;
+        if (it.n == 0) continue;
+        if (!it.src || !it.dst) return MXQ_ERR_NULL;
+        if (!aligned(it.src, 32) || !aligned(it.dst, 32)) return MXQ_ERR_ALIGN;
+    }
+    // launches of at most kFqBatchItemsMax tensors each: the item table rides in the kernel parameters
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<FqDeviceItem> chunk;
+    chunk.reserve(kFqBatchItemsMax);
+    size_t tiles = 0;
+    auto flush = [&]() -> int {
+        if (chunk.empty()) return MXQ_OK;
+        const int rc = launch_fake_quant_batched(chunk.data(), (int)chunk.size(), tiles, dtype, fmt, block, mode, s);
+        chunk.clear();
+        tiles = 0;
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const mxq_fq_item& it = items[i];
+        if (it.n == 0) continue;
+        FqDeviceItem d;
+        d.src = static_cast<const uint8_t*>(it.src);
+        d.dst = static_cast<uint8_t*>(it.dst);
+        d.nunits = it.n / epl;
+        d.tile_begin = tiles;
+        tiles += fq_batched_tiles(d.nunits);
+        chunk.push_back(d);
+        if ((int)chunk.size() == kFqBatchItemsMax)
+            if (int rc = flush()) return rc;
+    }
+    return flush();
+}
+
 int mxq_fake_quant_bwd(const void* grad_out, int dtype, size_t n, void* grad_in, mxq_stream stream)
 {
     if (!valid_dtype(dtype)) return MXQ_ERR_FORMAT;

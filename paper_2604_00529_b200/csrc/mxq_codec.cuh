@@ -110,28 +110,8 @@ __device__ __forceinline__ float scale_value(uint32_t byte)
 }
 
 // ------------------------------------------------------------------------------------------
-// Element quantizers (Eq. 2-3).  `v` is the raw element, `inv` = 2^-shared_exp; v * inv is exact.
+// MXFP element quantizers (Eq. 2).  `v` is the raw element, `inv` = 2^-shared_exp; v * inv is exact.
 // ------------------------------------------------------------------------------------------
-
-// MXINT magnitude: floor(|v| inv + 0.5), clipped to 2^(b-1)-1.
-// One FFMA rounded toward -inf adds 2^22 + 0.5, where the FP32 spacing is 0.5: the mantissa field
-// becomes floor(2 (|r| + 0.5)); halving it (floor) gives floor(|r| + 0.5) exactly.
-template <class F>
-__device__ __forceinline__ uint32_t int_magnitude(float v, float inv)
-{
-    constexpr float kMagic = 4194304.5f;
-    float y = __fmaf_rd(fabsf(v), inv, kMagic);
-    y = fminf(y, kMagic + (float)F::max_mag);
-    return (__float_as_uint(y) >> 1) & 0xFFu;
-}
-
-template <class F>
-__device__ __forceinline__ uint32_t quantize_int(float v, float inv)
-{
-    uint32_t q = int_magnitude<F>(v, inv);
-    uint32_t m = (uint32_t)((int32_t)__float_as_uint(v) >> 31);   // all ones for negative v
-    return ((q ^ m) - m) & F::mask;
-}
 
 // MXFP by plain ALU arithmetic, any (eta, mu): add 2^(ea + 23 - mu) so that the FP32 adder
 // rounds |r| (nearest even) to the element grid of its binade (ea = max(exponent, emin)); the
@@ -181,16 +161,14 @@ __device__ __forceinline__ uint32_t quantize_fp_hw_pair(float r0, float r1)
     return d;
 }
 
-// Quantize two scaled-on-the-fly elements; returns the two codes in the low `bits` bits of
-// .x and .y.
+// Quantize two scaled-on-the-fly elements to an MXFP format; returns the two codes in the low `bits`
+// bits of .x and .y.  (MXINT elements are quantized four at a time, see quantize_int_quad.)
 template <class F>
 __device__ __forceinline__ uint2 quantize_pair(float v0, float v1, float inv)
 {
+    static_assert(F::kind == KIND_FP, "MXFP formats only");
     uint2 c;
-    if constexpr (F::kind == KIND_INT) {
-        c.x = quantize_int<F>(v0, inv);
-        c.y = quantize_int<F>(v1, inv);
-    } else if constexpr (F::hw_cvt) {
+    if constexpr (F::hw_cvt) {
         uint32_t d = quantize_fp_hw_pair<F>(v0 * inv, v1 * inv);
         if constexpr (F::bits == 4) {
             c.x = d & 0xFu;

@@ -9,9 +9,10 @@
 //   slice_scale           : unit = 32 element codes = one block per lane, no cross-lane traffic.
 //   dequantize            : unit = 32 element codes in, 64 / 128 B out.
 //
-// All of them are bound by HBM traffic; the instruction budget per element is what the code
-// below is shaped around (packed 16-bit maxima, round-down FFMA instead of float->int
-// conversions, SWAR on four 8-bit codes per register, the sm_100a narrowing cvt instructions).
+// All of them are bound by HBM traffic, with the integer/logic pipe (64 lanes per clock per SM) as
+// the second bound; the arithmetic below is shaped to stay under it: packed 16-bit maxima, round-down
+// FP32 adds instead of float->int conversions, four 8-bit codes per register (SWAR), per-byte signs
+// by byte permutes and one multiply, the sm_100a narrowing conversion instructions for MXFP.
 #pragma once
 #include <cstdint>
 #include <utility>
@@ -339,69 +340,104 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return d;
 }
 
-template <class T, class F, int BLOCK, int MODE, int U, int THREADS>
-__global__ void __launch_bounds__(THREADS)
-fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may equal src
+// One warp tile (32 U lane units) of one tensor; shared by the single-tensor and the batched kernels.
+// Every lane of the warp must call it (the block maxima meet by shuffles).
+template <class T, class F, int BLOCK, int MODE, int U>
+__device__ __forceinline__ void fake_quant_tile(const uint8_t* src, size_t nunits, uint8_t* dst, size_t tile)
 {
-    pdl_release();
     using A = Fmt<F::kind == KIND_INT ? MXQ_INT8 : MXQ_FP8_E4M3>;
     constexpr bool via = MODE == MXQ_FQ_VIA_ANCHOR && F::id != A::id;
     using S = std::conditional_t<via, A, F>;            // the format whose scale Eq. 1 computes
     constexpr int de = A::emax - F::emax;
     constexpr int LPB = BLOCK / T::epl;
     static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
-    const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
-
-    pdl_acquire();
-    if (const size_t tile = warp; tile < ntiles) {
-        const size_t u0 = tile * (32 * U) + lane;
-        uint32_t w[U][8];
+    const size_t u0 = tile * (32 * U) + (threadIdx.x & 31);
+    uint32_t w[U][8];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit < nunits) ld256(w[u], src + unit * 32);
-            else {
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit < nunits) ld256(w[u], src + unit * 32);
+        else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) w[u][j] = 0;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
-            const BlockScale s = block_scale<S>(amax);
-            // X of the target format: the anchor's byte moved up by de, saturating (Eq. 4-5)
-            const uint32_t byte = via ? min(s.byte + (uint32_t)de, 254u) : s.byte;
-            const float X = scale_value(byte);
-            uint32_t out[8];
-            static_for<T::epl / 2>([&](auto i) {
-                constexpr int I = decltype(i)::value;
-                const float v0 = unit_elem<T, 2 * I>(w[u]), v1 = unit_elem<T, 2 * I + 1>(w[u]);
-                float2 p = fake_quant_pair<F, MODE>(v0, v1, s.inv);
-                float y0, y1;
-                if constexpr (F::kind == KIND_INT) {          // MXINT zero reconstructs to +0
-                    y0 = fma_keep_plus_zero(p.x, X);
-                    y1 = fma_keep_plus_zero(p.y, X);
-                } else {
-                    y0 = p.x * X;
-                    y1 = p.y * X;
-                }
-                if constexpr (T::size == 4) {
-                    out[2 * I] = __float_as_uint(y0);
-                    out[2 * I + 1] = __float_as_uint(y1);
-                } else {
-                    out[I] = pack_bf16x2(y0, y1);
-                }
-            });
-            if (s.byte == 0xFFu) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
-            }
-            if (unit < nunits) st256(dst + unit * 32, out);
+            for (int j = 0; j < 8; ++j) w[u][j] = 0;
         }
     }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
+        const BlockScale s = block_scale<S>(amax);
+        // X of the target format: the anchor's byte moved up by de, saturating (Eq. 4-5)
+        const uint32_t byte = via ? min(s.byte + (uint32_t)de, 254u) : s.byte;
+        const float X = scale_value(byte);
+        uint32_t out[8];
+        static_for<T::epl / 2>([&](auto i) {
+            constexpr int I = decltype(i)::value;
+            const float v0 = unit_elem<T, 2 * I>(w[u]), v1 = unit_elem<T, 2 * I + 1>(w[u]);
+            float2 p = fake_quant_pair<F, MODE>(v0, v1, s.inv);
+            float y0, y1;
+            if constexpr (F::kind == KIND_INT) {          // MXINT zero reconstructs to +0
+                y0 = fma_keep_plus_zero(p.x, X);
+                y1 = fma_keep_plus_zero(p.y, X);
+            } else {
+                y0 = p.x * X;
+                y1 = p.y * X;
+            }
+            if constexpr (T::size == 4) {
+                out[2 * I] = __float_as_uint(y0);
+                out[2 * I + 1] = __float_as_uint(y1);
+            } else {
+                out[I] = pack_bf16x2(y0, y1);
+            }
+        });
+        if (s.byte == 0xFFu) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+        }
+        if (unit < nunits) st256(dst + unit * 32, out);
+    }
+}
+
+template <class T, class F, int BLOCK, int MODE, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may equal src
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    pdl_acquire();
+    if (tile * (32 * U) < nunits) fake_quant_tile<T, F, BLOCK, MODE, U>(src, nunits, dst, tile);
+}
+
+// The fake-quant of a whole set of tensors (every quantized weight of a model in one QAT step, Eq. 6)
+// in one launch: the tiles of all tensors laid end to end, the item table in the kernel's parameters.
+struct FqDeviceItem {
+    const uint8_t* src;
+    uint8_t* dst;
+    size_t nunits;
+    size_t tile_begin;     // first global tile index of this tensor
+};
+
+template <int K>
+struct FqItemBlock {
+    FqDeviceItem items[K];
+};
+
+template <class T, class F, int BLOCK, int MODE, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS)
+fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count, size_t total_tiles)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    pdl_acquire();
+    if (tile >= total_tiles) return;                      // whole warps leave together
+    int lo = 0, hi = count - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (blk.items[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
+    }
+    const FqDeviceItem& t = blk.items[lo];
+    fake_quant_tile<T, F, BLOCK, MODE, U>(t.src, t.nunits, t.dst, tile - t.tile_begin);
 }
 
 // ------------------------------------------------------------------------------------------

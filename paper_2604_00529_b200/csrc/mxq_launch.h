@@ -32,6 +32,13 @@ int launch_slice_scale2(const void* codes, const uint8_t* scales, size_t n, int 
                         cudaStream_t stream);
 int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
                       cudaStream_t stream);
+// Fused fake-quant over up to kFqBatchItemsMax tensors in one launch; `items_host` is a HOST array
+// whose tile_begin fields are filled in.
+struct FqDeviceItem;
+constexpr int kFqBatchItemsMax = 512;
+int launch_fake_quant_batched(const FqDeviceItem* items_host, int count, size_t total_tiles, int dtype, int fmt,
+                              int block, int mode, cudaStream_t stream);
+size_t fq_batched_tiles(size_t nunits);
 int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
 
 // Batched Slice-and-Scale over a device-resident item table (see mxq_kernels.cuh: SsDeviceItem).

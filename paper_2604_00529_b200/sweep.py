@@ -140,6 +140,20 @@ def whole_model(reps: int = 5):
                                                   "elements": total, "tensors": len(items)}
             del oc, os_, table, items
         del codes, scales
+    # the QAT side of the same weight set: the fused fake-quant of all 224 BF16 weights (Eq. 6)
+    w = torch.randn(total, device="cuda", generator=g, dtype=torch.float32).mul_(0.02).to(torch.bfloat16)
+    y = torch.empty_like(w)
+    pairs, off = [], 0
+    for *_, r, c in shapes:
+        pairs.append((w[off:off + r * c], y[off:off + r * c]))
+        off += r * c
+    table = mxq.make_fq_items(pairs)
+    for fmt, mode, tag in (("e2m3", mxq.FQ_VIA_ANCHOR, "via_anchor"), ("int4", mxq.FQ_VIA_ANCHOR, "via_anchor")):
+        us = _time(lambda j: mxq.fake_quant_batched(table, fmt, BLOCK, mode), 1, reps)
+        per = _time(lambda j: [mxq.fake_quant(a, fmt, BLOCK, mode, dst=b) for a, b in pairs], 1, reps)
+        out["model_fake_quant_%s_%s" % (fmt, tag)] = {"batched_ms": us / 1e3, "batched_gbs": 4.0 * total / us / 1e3,
+                                                      "per_tensor_launches_ms": per / 1e3, "per_tensor_gbs": 4.0 * total / per / 1e3,
+                                                      "elements": total, "tensors": len(pairs)}
     return out
 
 

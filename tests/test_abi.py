@@ -87,6 +87,13 @@ def test_argument_checks_answer_on_the_host(L):
     fq = L.mxq_fake_quant
     assert fq(A, 1, 64, F["e2m1"], 32, 2, A, None) == E_FORMAT               # unknown mode
     assert fq(A, 1, 64, F["e2m1"], 32, 1, None, None) == E_NULL
+    fqb = L.mxq_fake_quant_batched
+    assert fqb(None, 0, 1, F["e2m1"], 32, 0, None) == OK
+    assert fqb(None, 3, 1, F["e2m1"], 32, 0, None) == E_NULL
+    assert fqb(None, -2, 1, F["e2m1"], 32, 0, None) == E_SIZE
+    assert fqb(None, 3, 1, F["e2m1"], 48, 0, None) == E_BLOCK
+    assert fqb(None, 3, 1, 77, 32, 0, None) == E_FORMAT
+    assert fqb(None, 3, 1, F["e2m1"], 32, 5, None) == E_FORMAT
     bw = L.mxq_fake_quant_bwd
     assert bw(A, 1, 64, A, None) == OK                                       # in place: no launch
     assert bw(A, 1, 64, None, None) == E_NULL
@@ -105,3 +112,35 @@ def test_binding_refuses_cpu_tensors():
         mxq.quantize(torch.zeros(64), "int8")
     with pytest.raises((TypeError, ValueError)):
         mxq.fake_quant(torch.zeros(64, dtype=torch.float16), "int8")
+
+
+def test_header_is_plain_c_and_links(tmp_path):
+    """include/mxq.h compiled as C99 by gcc, every declared function referenced, linked against libmxq.so
+    and run: the program only calls the size helpers and the host-side checks (no launch)."""
+    import subprocess
+    names = _declared_functions()
+    refs = "\n".join("    p[%d] = (fn)%s;" % (i, n) for i, n in enumerate(names))
+    src = tmp_path / "consumer.c"
+    src.write_text("""
+#include <stdio.h>
+#include "mxq.h"
+typedef void (*fn)(void);
+int main(void)
+{
+    fn p[%d];
+%s
+    for (int i = 0; i < %d; ++i) if (!p[i]) return 2;
+    if (mxq_format_bits(MXQ_FP6_E2M3) != 6 || mxq_codes_bytes(64, MXQ_INT4) != 32) return 3;
+    if (mxq_quantize(0, MXQ_BF16, 64, MXQ_INT8, 32, 0, 0, 0) != MXQ_ERR_NULL) return 4;
+    if (mxq_slice_scale(0, 0, 64, 32, MXQ_INT4, MXQ_INT8, 0, 0, 0) != MXQ_ERR_PAIR) return 5;
+    printf("%%s\\n", mxq_status_string(MXQ_ERR_PAIR));
+    return 0;
+}
+""" % (len(names), refs, len(names)))
+    exe = tmp_path / "consumer"
+    libdir = os.path.dirname(mxq.library_path())
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-l:libmxq.so", "-Wl,-rpath," + libdir])
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, (out.returncode, out.stderr)
+    assert "MXQ_ERR_PAIR" in out.stdout

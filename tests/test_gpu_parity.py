@@ -330,6 +330,32 @@ def test_fake_quant_in_place_and_backward():
     assert torch.equal(mxq.fake_quant_bwd(g32), g32)
 
 
+@pytest.mark.parametrize("count", [1, 7, 512, 513, 1100])
+@pytest.mark.parametrize("bf16", [True, False])
+def test_fake_quant_batched_matches_oracle(count, bf16):
+    """Many tensors of different sizes (down to one block) in one call, some of them in place; counts on
+    both sides of the 512-tensor launch limit."""
+    rng = np.random.default_rng(count)
+    nblks = rng.integers(1, 40, count)
+    if count <= 7:
+        nblks[0] = 3000                                          # one tensor of many tiles
+    fmt, mode = ("e2m3", orc.FQ_VIA_ANCHOR) if bf16 else ("int4", orc.FQ_DIRECT)
+    pairs, wants = [], []
+    for k, nb in enumerate(nblks):
+        x = _mixed_f32(int(nb), 1000 + k)
+        if bf16:
+            x = inputs.to_bf16_bits(x)
+        src = to_dev(x)
+        dst = None if k % 3 == 0 else torch.full_like(src, 7.0)
+        pairs.append((src, dst))
+        wants.append(orc.fake_quant(x, fmt, mode=mode))
+    mxq.fake_quant_batched(pairs, fmt, 32, mode)
+    torch.cuda.synchronize()
+    for (src, dst), want in zip(pairs, wants):
+        got = to_host(dst if dst is not None else src)
+        assert bits_equal(got, want), first_diff(got, want)
+
+
 # ---------------------------------------------------------------------------------------------
 # chained entry points and degenerate sizes
 # ---------------------------------------------------------------------------------------------
