@@ -2,7 +2,7 @@
 
     python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--json out.json]
 
-For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
+`--graph` times CUDA-graph replays instead of direct launches.  For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
 for every anchor-to-lower pair, reconstruction and the fused fake-quant, timed with CUDA events over
 back-to-back launches that rotate over enough buffer copies to exceed the 126 MB L2 (small sizes
 therefore show launch-bound, not cache-resident, figures).  GB/s counts algorithmic bytes (read +
@@ -33,8 +33,30 @@ def _peak():
         return 6650.0, "fallback"
 
 
+GRAPH = False     # --graph: time the replay of a CUDA graph that holds the launches (no host cost per launch)
+
+
 def _time(launch, copies: int, reps: int) -> float:
     """Average microseconds per launch; launch(j) must use buffer copy j."""
+    if GRAPH:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for j in range(min(3, copies)):
+                launch(j)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(reps):
+                launch(i % copies)
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / reps
     for j in range(min(3, copies)):
         launch(j)
     torch.cuda.synchronize()
@@ -163,11 +185,16 @@ def main():
     ap.add_argument("--max-log2", type=int, default=31)
     ap.add_argument("--model", action="store_true")
     ap.add_argument("--json", default=None)
+    ap.add_argument("--graph", action="store_true",
+                    help="capture each timed loop in a CUDA graph and time its replay: the figures then exclude the "
+                         "host's cost of enqueuing a launch (about 8 us through this binding)")
     args = ap.parse_args()
+    global GRAPH
+    GRAPH = args.graph
     mxq.load_library()
     peak, kind = _peak()
     base = torch.from_numpy(inputs.flat_bf16_normal(1 << 27, seed=5).view(np.int16)).cuda().view(torch.bfloat16)
-    result = {"peak_gbs": peak, "peak_kind": kind, "sizes": {}, "f32": {}, "model": {}}
+    result = {"peak_gbs": peak, "peak_kind": kind, "graph": GRAPH, "sizes": {}, "f32": {}, "model": {}}
     for k in range(args.min_log2, args.max_log2 + 1):
         n = 1 << k
         reps = 200 if k <= 22 else (50 if k <= 27 else 10)
