@@ -18,6 +18,11 @@
  *     global accesses); scale buffers must be 16-byte aligned.  The library enqueues work on
  *     `stream` and returns without synchronising.  Unless an entry point says otherwise it
  *     allocates nothing.
+ *   - Work goes to the CURRENT device, which must be the one the pointers belong to.  Kernels
+ *     are launched with programmatic stream serialization allowed, so that a kernel's blocks
+ *     can become resident while the previous kernel of the stream drains; each kernel waits
+ *     for that previous kernel to complete before its first global memory access, so the
+ *     ordering a stream guarantees is unchanged for every buffer.
  *   - `n` is the number of elements; it must be a multiple of `block`.  Blocks are runs
  *     of `block` consecutive elements of the flat array (for a row-major matrix whose inner
  *     dimension is a multiple of `block`: along the row).  n == 0 returns MXQ_OK at once.
