@@ -26,6 +26,8 @@
  *   - `n` is the number of elements; it must be a multiple of `block`.  Blocks are runs
  *     of `block` consecutive elements of the flat array (for a row-major matrix whose inner
  *     dimension is a multiple of `block`: along the row).  n == 0 returns MXQ_OK at once.
+ *     The entry points that read packed codes (mxq_slice_scale and its multi / batched forms,
+ *     mxq_dequantize) also need n to be a multiple of 32, which only matters for block 16.
  *   - The return value is an mxq_status.  Errors detectable on the host (bad enum, null
  *     or misaligned pointer, bad size) are reported before anything is launched;
  *     MXQ_ERR_CUDA reports a failed launch (cudaGetLastError()).
