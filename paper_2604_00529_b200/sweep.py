@@ -109,7 +109,8 @@ def sweep_size(n: int, base_dev: torch.Tensor, reps: int):
     rec("slice_scale_multi_e4m3_e2m3+e2m1", us, 1 + 6 / 8 + 4 / 8 + 3 / BLOCK)
     del two, anchors
     ys = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
-    for fmt, mode, tag in (("e2m3", mxq.FQ_VIA_ANCHOR, "via_anchor"), ("int4", mxq.FQ_DIRECT, "direct")):
+    for fmt, mode, tag in (("e2m3", mxq.FQ_VIA_ANCHOR, "via_anchor"), ("int4", mxq.FQ_DIRECT, "direct"),
+                           ("int4", mxq.FQ_VIA_ANCHOR, "via_anchor"), ("e2m1", mxq.FQ_VIA_ANCHOR, "via_anchor")):
         us = _time(lambda j: mxq.fake_quant(xs[j], fmt, BLOCK, mode, dst=ys[j]), copies, reps)
         rec("fake_quant_bf16_%s_%s" % (fmt, tag), us, 4.0)
     return out, copies

@@ -189,7 +189,8 @@ def w5_base():
     return inputs.flat_bf16_normal(_W5_BASE, seed=5)
 
 
-@pytest.mark.parametrize("log2n", [16, 20, 24, 28, 31])
+@pytest.mark.parametrize("log2n", [16, 20, 24, 28, 31, 33])     # 33: beyond the listed sizes, element and byte
+                                                                     # offsets past 2^32
 def test_workload5_size_sweep(w5_base, log2n):
     n = 1 << log2n
     base = w5_base

@@ -419,3 +419,30 @@ def test_tensor_level_mse_study_on_gpu():
         by_block.append((mse(d), mse(s)))
     assert all(a[0] < b[0] and a[1] < b[1] for a, b in zip(by_block[:-1], by_block[1:]))   # smaller blocks, lower error
     assert all(1.0 <= s / d < 1.2 for d, s in by_block)
+
+
+def test_two_streams_run_independent_conversions():
+    """The same calls issued on two non-default streams at once give what they give alone (every
+    entry point takes its stream from the caller; only the >512-tensor batched path shares state)."""
+    x1 = inputs.to_bf16_bits(_mixed_f32(4099, 21))
+    x2 = inputs.to_bf16_bits(_mixed_f32(4099, 22))
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    d1, d2 = to_dev(x1), to_dev(x2)
+    torch.cuda.synchronize()
+    res = {}
+    for rep in range(3):
+        for name, st, d, fmt, low in (("a", s1, d1, "e4m3", "e2m1"), ("b", s2, d2, "int8", "int6")):
+            with torch.cuda.stream(st):
+                c, s = mxq.quantize(d, fmt)
+                lc, ls = mxq.slice_scale(c, s, d.numel(), fmt, low)
+                v = mxq.dequantize(lc, ls, d.numel(), low, dtype=torch.bfloat16)
+                y = mxq.fake_quant(d, low, mode=mxq.FQ_VIA_ANCHOR)
+                res[name] = (lc, ls, v, y)
+    torch.cuda.synchronize()
+    for name, x, fmt, low in (("a", x1, "e4m3", "e2m1"), ("b", x2, "int8", "int6")):
+        lc, ls, v, y = res[name]
+        oc, os_ = orc.quantize(x, fmt)
+        wc, ws = orc.slice_scale(oc, os_, fmt, low)
+        assert bits_equal(to_host(lc), orc.pack(wc, orc.bits(low))) and bits_equal(to_host(ls), ws)
+        assert bits_equal(to_host(v), orc.dequantize(wc, ws, low, out_dtype=orc.BF16))
+        assert bits_equal(to_host(y), orc.fake_quant(x, low, mode=orc.FQ_VIA_ANCHOR))
