@@ -139,6 +139,35 @@ __device__ __forceinline__ void store_bytes(void* p, const uint32_t (&w)[NW])
     }
 }
 
+// ---- staged tile stores ------------------------------------------------------------------------
+// A lane's piece of packed codes is OB bytes at lane * OB of its warp tile.  When OB is not one
+// aligned vector a direct store takes several narrow instructions, each of which touches every
+// 32-byte sector of the tile with a few bytes.  For the 7-bit formats that is seven 2- or 4-byte
+// stores per lane (measured 3.0 - 3.5 TB/s); their tiles go through shared memory instead: lanes
+// drop their pieces there and the warp copies the tile out as 16-byte pieces in address order
+// (5.4 TB/s).  With five or fewer direct stores (24, 20, 12, 10, 6 bytes) staging measured slower
+// than storing directly, so those keep the direct path.
+
+// store instructions a lane needs for a direct store of OB bytes
+__host__ __device__ constexpr int direct_store_count(int bytes) { return bytes / piece_align(bytes); }
+
+template <int OB>
+struct StagedTile {
+    static constexpr bool use = direct_store_count(OB) > 5;
+};
+
+// Copy the first `nbytes` bytes of a warp's staging area to `gdst` (16-byte aligned, like the area).
+__device__ __forceinline__ void flush_stage(const uint8_t* stage, uint8_t* gdst, uint32_t nbytes)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    __syncwarp();
+    for (uint32_t i = lane * 16; i + 16 <= nbytes; i += 512)
+        *reinterpret_cast<uint4*>(gdst + i) = *reinterpret_cast<const uint4*>(stage + i);
+    const uint32_t done = nbytes & ~15u;                        // a ragged tensor end: up to 15 bytes
+    if (done + lane < nbytes) gdst[done + lane] = stage[done + lane];
+    __syncwarp();
+}
+
 // ---- bitstream of element codes in registers -------------------------------------------------
 
 // Words needed for N codes of BITS bits.

@@ -113,6 +113,35 @@ __device__ __forceinline__ void join24(uint32_t z0, uint32_t z1, uint32_t z2, ui
     o2 = (z2 >> 16) | (z3 << 8);
 }
 
+// Four B-bit codes, one per byte with the upper bits clear, -> one 4B-bit value (c0 | c1 << B | ...).
+// Two shift-and-select steps: bytes to 2B-bit fields in the 16-bit halves, halves to one field.
+// Whatever a shift drags along falls where the next select takes the other operand.
+template <int B>
+__device__ __forceinline__ uint32_t squeeze_bytes(uint32_t x)
+{
+    static_assert(B >= 1 && B <= 7, "codes narrower than a byte");
+    constexpr uint32_t kEven = ((1u << B) - 1u) * 0x00010001u;           // the fields of bytes 0 and 2
+    constexpr uint32_t kLow = (1u << (2 * B)) - 1u;
+    const uint32_t y = (x & kEven) | ((x >> (8 - B)) & ~kEven);
+    return (y & kLow) | ((y >> (16 - 2 * B)) & ~kLow);
+}
+
+// NZ words holding four clean B-bit codes each (one per byte) -> the little-endian bitstream.
+template <int B, int NZ, int NW>
+__device__ __forceinline__ void pack_code_bytes(const uint32_t (&z)[NZ], uint32_t (&out)[NW])
+{
+    constexpr int W = 4 * B;                                             // bits per squeezed word
+    static_assert(NW * 32 >= NZ * W, "output too small");
+    static_for<NZ>([&](auto j) {
+        constexpr int J = decltype(j)::value;
+        constexpr int off = J * W, wi = off >> 5, sh = off & 31;
+        const uint32_t q = squeeze_bytes<B>(z[J]);
+        if constexpr (sh == 0) out[wi] = q;
+        else out[wi] |= q << sh;
+        if constexpr (sh + W > 32) out[wi + 1] = q >> (32 - sh);
+    });
+}
+
 // MXINT codes of four consecutive elements (Eq. 3), one per byte in the low F::bits bits.
 //   v0..v3 : the raw elements, inv = 2^-shared_exp (|v| inv < 2^(bits-1), exact)
 //   full   : 0xFF in the bytes whose element is negative, 0x00 elsewhere
@@ -186,10 +215,7 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
                 join24(s0, s1, s2, s3, out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
             }
         } else {
-            static_for<T::epl>([&](auto i) {
-                constexpr int I = decltype(i)::value;
-                put_code<F::bits, I>(out, (z[I / 4] >> (8 * (I % 4))) & F::mask);
-            });
+            pack_code_bytes<F::bits>(z, out);
         }
     } else {
         static_for<T::epl / 2>([&](auto i) {
@@ -222,6 +248,11 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    uint8_t* stage = nullptr;
+    if constexpr (StagedTile<OB>::use) {
+        __shared__ __align__(16) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
+        stage = stage_area + (threadIdx.x >> 5) * (32 * U * OB);
+    }
 
     pdl_acquire();
     if (const size_t tile = warp; tile < ntiles) {
@@ -247,10 +278,15 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
 #pragma unroll
                 for (int j = 0; j < NW; ++j) out[j] = 0;
             }
+            if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + lane) * OB, out);
             if (unit < nunits) {
-                store_bytes<OB>(codes + unit * OB, out);
+                if constexpr (!StagedTile<OB>::use) store_bytes<OB>(codes + unit * OB, out);
                 if (lane % LPB == 0) scales[unit / LPB] = (uint8_t)s.byte;
             }
+        }
+        if constexpr (StagedTile<OB>::use) {
+            const size_t first = tile * (32 * U), left = nunits - first;
+            flush_stage(stage, codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
         }
     }
 }
@@ -545,6 +581,12 @@ __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint
         for (int g = 0; g < 2; ++g) {
             join24(z[4 * g + 0], z[4 * g + 1], z[4 * g + 2], z[4 * g + 3], out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
         }
+    } else if constexpr (FH::id == MXQ_INT8 && FL::kind == KIND_INT) {
+        // MXINT7 / 5 / 3 / 2: the same four-codes-per-register arithmetic, generic packing
+        uint32_t z[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) z[j] = ss_int8_word<FL::bits>(in[j]);
+        pack_code_bytes<FL::bits>(z, out);
     } else if constexpr (FH::id == MXQ_FP8_E4M3 && FL::hw_cvt) {
         bool nan = false;
 #pragma unroll
@@ -597,7 +639,7 @@ __device__ __forceinline__ uint8_t ss_scale_byte(uint32_t b, int de)
 template <class FH, class FL, int U>
 __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
                                                  size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
-                                                 uint8_t* __restrict__ out_scales, size_t tile)
+                                                 uint8_t* __restrict__ out_scales, size_t tile, uint8_t* stage)
 {
     constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;      // bytes per lane unit
     constexpr int NWI = IB / 4, NWO = OB / 4;
@@ -621,7 +663,12 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
         if (unit < nscales) out_scales[unit] = ss_scale_byte(sb[u], de);
         uint32_t out[NWO];
         slice_scale_unit<FH, FL>(w[u], out);
-        if (unit < nunits) store_bytes<OB>(out_codes + unit * OB, out);
+        if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + (threadIdx.x & 31)) * OB, out);
+        else if (unit < nunits) store_bytes<OB>(out_codes + unit * OB, out);
+    }
+    if constexpr (StagedTile<OB>::use) {
+        const size_t first = tile * (32 * U), left = nunits - first;
+        flush_stage(stage, out_codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
     }
     if (nscales > nunits) {
 #pragma unroll
@@ -632,6 +679,20 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
     }
 }
 
+// The staging area of the calling warp for a Slice-and-Scale tile (null when the target's pieces are
+// single vectors).  Must be called by every thread of the CTA, outside divergent code.
+template <class FL, int U, int THREADS>
+__device__ __forceinline__ uint8_t* slice_scale_stage()
+{
+    constexpr int OB = 4 * FL::bits;
+    if constexpr (StagedTile<OB>::use) {
+        __shared__ __align__(16) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
+        return stage_area + (threadIdx.x >> 5) * (32 * U * OB);
+    } else {
+        return nullptr;
+    }
+}
+
 template <class FH, class FL, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
@@ -639,8 +700,10 @@ slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
     pdl_acquire();
-    if (tile * (32 * U) < nunits) slice_scale_tile<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, tile);
+    if (tile * (32 * U) < nunits)
+        slice_scale_tile<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, tile, stage);
 }
 
 // Two targets from one read of the anchor (the elastic-serving case: one stored checkpoint, several
@@ -657,7 +720,18 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
     constexpr int de1 = FH::emax - FL1::emax, de2 = FH::emax - FL2::emax;
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t u0 = tile * (32 * U) + (threadIdx.x & 31);
+    uint8_t* stage1 = nullptr;
+    uint8_t* stage2 = nullptr;
+    if constexpr (StagedTile<OB1>::use) {
+        __shared__ __align__(16) uint8_t area1[(THREADS / 32) * 32 * U * OB1];
+        stage1 = area1 + (threadIdx.x >> 5) * (32 * U * OB1);
+    }
+    if constexpr (StagedTile<OB2>::use) {
+        __shared__ __align__(16) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
+        stage2 = area2 + (threadIdx.x >> 5) * (32 * U * OB2);
+    }
     pdl_acquire();
+    if (tile * (32 * U) >= nunits) return;                     // whole warps leave together
     uint32_t w[U][NWI];
     uint32_t sb[U];
 #pragma unroll
@@ -679,9 +753,17 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
         }
         uint32_t o1[OB1 / 4], o2[OB2 / 4];
         slice_scale_unit<FH, FL1>(w[u], o1);
-        if (unit < nunits) store_bytes<OB1>(out_codes1 + unit * OB1, o1);
+        if constexpr (StagedTile<OB1>::use) store_bytes<OB1>(stage1 + (u * 32 + (threadIdx.x & 31)) * OB1, o1);
+        else if (unit < nunits) store_bytes<OB1>(out_codes1 + unit * OB1, o1);
         slice_scale_unit<FH, FL2>(w[u], o2);
-        if (unit < nunits) store_bytes<OB2>(out_codes2 + unit * OB2, o2);
+        if constexpr (StagedTile<OB2>::use) store_bytes<OB2>(stage2 + (u * 32 + (threadIdx.x & 31)) * OB2, o2);
+        else if (unit < nunits) store_bytes<OB2>(out_codes2 + unit * OB2, o2);
+    }
+    {
+        const size_t first = tile * (32 * U), left = nunits - first;
+        const uint32_t valid = (uint32_t)(left < 32 * U ? left : 32 * U);
+        if constexpr (StagedTile<OB1>::use) flush_stage(stage1, out_codes1 + first * OB1, valid * OB1);
+        if constexpr (StagedTile<OB2>::use) flush_stage(stage2, out_codes2 + first * OB2, valid * OB2);
     }
     if (nscales > nunits) {
 #pragma unroll
@@ -717,6 +799,7 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
     pdl_acquire();
     if (tile >= total_tiles) return;
     // items are sorted by tile_begin: the last one that starts at or before this tile owns it
@@ -727,7 +810,8 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
         else hi = mid - 1;
     }
     const SsDeviceItem t = items[lo];
-    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin);
+    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin,
+                                stage);
 }
 
 // The same launch with the item table carried in the kernel's parameter space (K items, 56 bytes
@@ -744,6 +828,7 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
     pdl_acquire();
     if (tile >= total_tiles) return;
     int lo = 0, hi = count - 1;
@@ -753,7 +838,8 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
         else hi = mid - 1;
     }
     const SsDeviceItem& t = blk.items[lo];
-    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin);
+    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin,
+                                stage);
 }
 
 // ------------------------------------------------------------------------------------------
