@@ -558,6 +558,50 @@ __device__ __forceinline__ uint32_t ss_e4m3_words_to_e2m1(uint32_t w0, uint32_t 
     return d;
 }
 
+// Eq. 5 for the two MXFP targets without a narrowing instruction, E3M3 (7 bits, de = 4) and E2M2
+// (5 bits, de = 6), on four E4M3 codes per register (no NaN codes among them).  Two facts do the work:
+//   - where the result is a normal number of the target, it follows from the anchor's magnitude
+//     code by integer arithmetic: E3M3 keeps the three mantissa bits (code - 64); E2M2 drops one
+//     (code / 2 rounded half to even, minus 48);
+//   - everywhere else the target's grid is uniform with step 2^-5 (E3M3) or 2^-2 (E2M2), and the
+//     magnitude code of k steps is k itself up to the second binade.  k = RNE(|v| / 16) for both, one
+//     FP16 fused multiply-add per pair of codes: |v| / 16 + C with C = 32 (step 2^-5... in units of
+//     the divided value) or 1024 (step 1) leaves k in the low mantissa bits of the sum.
+// The two regimes agree on the codes where they meet, so a per-byte threshold selects between them.
+template <class FL>
+__device__ __forceinline__ uint32_t ss_e4m3_word_soft(uint32_t x)
+{
+    static_assert(FL::id == MXQ_FP7_E3M3 || FL::id == MXQ_FP5_E2M2, "E3M3 or E2M2");
+    constexpr bool e3m3 = FL::id == MXQ_FP7_E3M3;
+    constexpr uint32_t k01 = 0x01010101u;
+    const uint32_t mag = x & 0x7F7F7F7Fu;
+    // k for the four codes: FP16 pairs, |v| * 2^-4 + C, low byte of each half
+    constexpr uint32_t kSixteenth = 0x2C002C00u;                        // 2^-4 as FP16 x2
+    constexpr uint32_t kC = e3m3 ? 0x50005000u : 0x64006400u;           // 32.0 / 1024.0 as FP16 x2
+    uint32_t a, b;
+    asm("{ .reg .b16 l, h;\n"
+        "  mov.b32 {l, h}, %2;\n"
+        "  cvt.rn.f16x2.e4m3x2 %0, l;  cvt.rn.f16x2.e4m3x2 %1, h;\n"
+        "  fma.rn.f16x2 %0, %0, %3, %4;  fma.rn.f16x2 %1, %1, %3, %4; }"
+        : "=r"(a), "=r"(b) : "r"(mag), "r"(kSixteenth), "r"(kC));
+    const uint32_t k = __byte_perm(a, b, 0x6420);
+    // the normal regime, valid from code kFrom on
+    constexpr uint32_t kFrom = e3m3 ? 72u : 104u;
+    uint32_t normal;
+    if constexpr (e3m3) {
+        normal = mag & 0x3F3F3F3Fu;                                      // code - 64 for codes >= 64
+    } else {
+        const uint32_t q = (mag >> 1) & 0x3F3F3F3Fu;
+        const uint32_t t = q + (mag & q & k01);                          // code / 2, ties to even: 52 .. 63
+        normal = t & 0x0F0F0F0Fu;                                        // - 48
+    }
+    uint32_t full;                                                       // 0xFF where code >= kFrom
+    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(mag + k01 * (128u - kFrom)));
+    const uint32_t m = (normal & full) | (k & ~full);
+    constexpr int sh = 8 - FL::bits;                                     // sign: bit 7 -> bit (bits - 1)
+    return m | ((x >> sh) & (k01 << (FL::bits - 1)));
+}
+
 // Convert the 32 codes of one lane.  in: 8*FH::bits/8... words of the high format's bitstream.
 template <class FH, class FL, int NWI, int NWO>
 __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint32_t (&out)[NWO])
@@ -609,6 +653,21 @@ __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint
             // an E4M3 NaN code (never produced by the quantizer): exact scalar path
 #pragma unroll
             for (int j = 0; j < NWO; ++j) out[j] = 0;
+            static_for<32>([&](auto i) {
+                constexpr int I = decltype(i)::value;
+                put_code<FL::bits, I>(out, ss_fp_elem<FH, FL>(get_code<FH::bits, I>(in)));
+            });
+        }
+    } else if constexpr (FH::id == MXQ_FP8_E4M3 && (FL::id == MXQ_FP7_E3M3 || FL::id == MXQ_FP5_E2M2)) {
+        bool nan = false;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) nan |= has_e4m3_nan(in[j]);
+        if (!nan) {
+            uint32_t z[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) z[j] = ss_e4m3_word_soft<FL>(in[j]);
+            pack_code_bytes<FL::bits>(z, out);
+        } else {
             static_for<32>([&](auto i) {
                 constexpr int I = decltype(i)::value;
                 put_code<FL::bits, I>(out, ss_fp_elem<FH, FL>(get_code<FH::bits, I>(in)));
