@@ -217,6 +217,16 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
         } else {
             pack_code_bytes<F::bits>(z, out);
         }
+    } else if constexpr (!F::hw_cvt) {
+        // E3M3 / E2M2: four elements at a time through the hardware neighbour format
+        constexpr int NQ = T::epl / 4;
+        uint32_t z[NQ];
+        static_for<NQ>([&](auto qi) {
+            constexpr int Q = decltype(qi)::value;
+            z[Q] = quantize_fp_soft_quad<F>(unit_elem<T, 4 * Q>(w) * inv, unit_elem<T, 4 * Q + 1>(w) * inv,
+                                            unit_elem<T, 4 * Q + 2>(w) * inv, unit_elem<T, 4 * Q + 3>(w) * inv);
+        });
+        pack_code_bytes<F::bits>(z, out);
     } else {
         static_for<T::epl / 2>([&](auto i) {
             constexpr int I = decltype(i)::value;
@@ -362,8 +372,10 @@ __device__ __forceinline__ float2 fake_quant_pair(float v0, float v1, float inv)
         if constexpr (F::hw_cvt) {
             p = widen_hw_pair<F>(quantize_fp_hw_pair<F>(r0, r1));
         } else {
-            p.x = decode<F>(quantize_fp_alu<F>(r0));
-            p.y = decode<F>(quantize_fp_alu<F>(r1));
+            using N = Fmt<SoftFp<F>::hw>;
+            const float2 n = widen_hw_pair<N>(quantize_fp_hw_pair<N>(r0, r1));
+            p.x = quantize_fp_soft_value<F>(r0, n.x);
+            p.y = quantize_fp_soft_value<F>(r1, n.y);
         }
     }
     return p;
