@@ -1,6 +1,6 @@
 """Bandwidth sweep of libmxq on one GPU.
 
-    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--json out.json]
+    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--all-formats] [--graph] [--json out.json]
 
 `--graph` times CUDA-graph replays instead of direct launches.  For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
 for every anchor-to-lower pair, reconstruction and the fused fake-quant, timed with CUDA events over
@@ -135,6 +135,39 @@ def sweep_f32(n: int, reps: int):
     return out
 
 
+def all_formats(n: int, reps: int = 20):
+    """Every element format of the paper (MXINT2..8, MXFP4..8) at one size: Slice-and-Scale from the
+    anchor, direct quantization, reconstruction and the fused fake-quant through the anchor."""
+    bits = {"int8": 8, "int7": 7, "int6": 6, "int5": 5, "int4": 4, "int3": 3, "int2": 2,
+            "e4m3": 8, "e3m3": 7, "e3m2": 6, "e2m3": 6, "e2m2": 5, "e2m1": 4}
+    g = torch.Generator(device="cuda").manual_seed(1)
+    copies = 4
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    codes = [torch.randint(0, 127, (n,), generator=g, **u8) for _ in range(copies)]           # no E4M3 NaN codes
+    scales = [torch.randint(100, 140, (n // BLOCK,), generator=g, **u8) for _ in range(copies)]
+    x = [torch.randn(n, device="cuda", generator=g).to(torch.bfloat16) for _ in range(copies)]
+    y = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+    out = {}
+    for src, dsts in (("int8", ("int7", "int6", "int5", "int4", "int3", "int2")),
+                      ("e4m3", ("e3m3", "e3m2", "e2m3", "e2m2", "e2m1"))):
+        for d in dsts:
+            b = bits[d]
+            oc = [torch.empty(n * b // 8, **u8) for _ in range(copies)]
+            os_ = [torch.empty(n // BLOCK, **u8) for _ in range(copies)]
+            row = {}
+            us = _time(lambda j: mxq.slice_scale(codes[j], scales[j], n, src, d, BLOCK, oc[j], os_[j]), copies, reps)
+            row["slice_scale_from_anchor"] = (us, n * (1 + b / 8 + 2 / BLOCK) / us / 1e3)
+            us = _time(lambda j: mxq.quantize(x[j], d, BLOCK, oc[j], os_[j]), copies, reps)
+            row["quantize_bf16"] = (us, n * (2 + b / 8 + 1 / BLOCK) / us / 1e3)
+            us = _time(lambda j: mxq.dequantize(oc[j], os_[j], n, d, BLOCK, dst=y[j]), copies, reps)
+            row["dequantize_bf16"] = (us, n * (2 + b / 8 + 1 / BLOCK) / us / 1e3)
+            us = _time(lambda j: mxq.fake_quant(x[j], d, BLOCK, mxq.FQ_VIA_ANCHOR, dst=y[j]), copies, reps)
+            row["fake_quant_bf16_via_anchor"] = (us, n * 4.0 / us / 1e3)
+            out[d] = row
+            del oc, os_
+    return out
+
+
 def whole_model(reps: int = 5):
     """Anchor -> target for the 224 tensors of the 8B Llama-shaped set, one batched launch per target.
     Anchors hold seeded random codes (the conversion's speed does not depend on the values)."""
@@ -185,6 +218,7 @@ def main():
     ap.add_argument("--min-log2", type=int, default=16)
     ap.add_argument("--max-log2", type=int, default=31)
     ap.add_argument("--model", action="store_true")
+    ap.add_argument("--all-formats", action="store_true", help="every element format of the paper at 2^26 elements")
     ap.add_argument("--json", default=None)
     ap.add_argument("--graph", action="store_true",
                     help="capture each timed loop in a CUDA graph and time its replay: the figures then exclude the "
@@ -210,6 +244,13 @@ def main():
     print("FP32 entry points, 2^26 elements")
     for name, (us, g) in f32.items():
         print("  %-36s %10.2f us %8.1f GB/s  %5.1f %% of %s peak" % (name, us, g, 100 * g / peak, kind))
+    if args.all_formats:
+        fm = all_formats(1 << 26)
+        result["formats"] = {f: {op: {"us": round(us, 3), "gbs": round(g, 1)} for op, (us, g) in row.items()}
+                             for f, row in fm.items()}
+        print("all formats, 2^26 elements: GB/s (us)")
+        for f, row in fm.items():
+            print("  %-5s " % f + "  ".join("%s %6.0f (%5.1f)" % (op, g, us) for op, (us, g) in row.items()))
     if args.model:
         result["model"] = whole_model()
         for name, r in result["model"].items():
