@@ -19,8 +19,10 @@ import threading
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "mxq_oracle.c")
-_LIB = os.path.join(_HERE, "libmxq_oracle.so")
+# MXQ_ORACLE_SOURCE points the front end at another C file (the mutation test compiles copies of the
+# oracle with one planted mistake each and checks that the pins catch it); its library is built beside it.
+_SRC = os.environ.get("MXQ_ORACLE_SOURCE") or os.path.join(_HERE, "mxq_oracle.c")
+_LIB = os.path.join(os.path.dirname(os.path.abspath(_SRC)), "libmxq_oracle.so")
 
 F32, BF16 = 0, 1
 FQ_DIRECT, FQ_VIA_ANCHOR = 0, 1
