@@ -343,14 +343,17 @@ __device__ __forceinline__ float2 fake_quant_pair(float v0, float v1, float inv)
         // on the 0.5 grid of [2^22, 2^23), a round-down add of another 2^22 on the integer grid of
         // [2^23, 2^24).  The value stays biased by 2^23 until the clip.
         auto one = [&](float v) {
-            float z = __fadd_rd(__fmaf_rd(fabsf(v), inv, 4194304.5f), 4194304.0f);     // 2^23 + floor(|r| + 0.5)
+            float y = __fmaf_rd(fabsf(v), inv, 4194304.5f);                            // 2^22 + h, h = |r| + 0.5 on the 0.5 grid
             if constexpr (via) {
-                // Eq. 4 on the anchor magnitude q8 = z - 2^23: floor(q8 / 2^de + 0.5), the same way.
-                // (Clipping q8 to 127 first would change nothing: 127 and 128 both end in the clipped bin.)
+                // Eq. 4 on the anchor magnitude q8 = floor(h): floor(q8 / 2^de + 0.5) = floor(h / 2^de + 0.5),
+                // since flooring before a division by an integer changes nothing.  So the anchor's integer
+                // step is skipped: one more round-down multiply-add onto the 0.5 grid.
+                // (Clipping q8 to 127 first would change nothing either: 127 and 128 both end in the clipped bin.)
                 constexpr float kScale = 1.0f / (float)(1 << de);
-                constexpr float kBias = 4194304.5f - 8388608.0f / (float)(1 << de);    // exact in FP32
-                z = __fadd_rd(__fmaf_rd(z, kScale, kBias), 4194304.0f);
+                constexpr float kBias = 4194304.5f - 4194304.0f / (float)(1 << de);    // exact in FP32
+                y = __fmaf_rd(y, kScale, kBias);
             }
+            float z = __fadd_rd(y, 4194304.0f);                                        // 2^23 + floor(.)
             z = fminf(z, 8388608.0f + (float)F::max_mag);                              // symmetric clip
             const float qf = z - 8388608.0f;                                           // exact small integer
             return __uint_as_float(__float_as_uint(qf) | (__float_as_uint(v) & 0x80000000u));
