@@ -527,18 +527,26 @@ __device__ __forceinline__ bool has_e4m3_nan(uint32_t x)
 // by 2^de, FP32, narrowing cvt (nearest even, saturating).  Register halves and bytes are split and
 // joined with mov so that no shift or mask is spent on them.
 
+// four E4M3 codes of one word as two FP16 pairs (exact).  Kept apart from the scaling so that two
+// targets converted from the same word share it.
+__device__ __forceinline__ void e4m3_word_to_f16(uint32_t w, uint32_t& a, uint32_t& b)
+{
+    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.rn.f16x2.e4m3x2 %0, l; cvt.rn.f16x2.e4m3x2 %1, h; }"
+        : "=r"(a), "=r"(b) : "r"(w));
+}
+
 // two FP16 pairs (four E4M3 codes of one word), already divided by 2^de, as four FP32 values
 template <int DE>
 __device__ __forceinline__ void e4m3_word_scaled(uint32_t w, float (&f)[4])
 {
     constexpr uint32_t kHalf = (uint32_t)(15 - DE) << 10;      // 2^-de as FP16
+    uint32_t a, b;
+    e4m3_word_to_f16(w, a, b);
     asm("{ .reg .b16 l, h; .reg .b32 a, b;\n"
-        "  mov.b32 {l, h}, %4;\n"
-        "  cvt.rn.f16x2.e4m3x2 a, l;  cvt.rn.f16x2.e4m3x2 b, h;\n"
-        "  mul.rn.f16x2 a, a, %5;  mul.rn.f16x2 b, b, %5;\n"
+        "  mul.rn.f16x2 a, %4, %6;  mul.rn.f16x2 b, %5, %6;\n"
         "  mov.b32 {l, h}, a;  cvt.f32.f16 %0, l;  cvt.f32.f16 %1, h;\n"
         "  mov.b32 {l, h}, b;  cvt.f32.f16 %2, l;  cvt.f32.f16 %3, h; }"
-        : "=f"(f[0]), "=f"(f[1]), "=f"(f[2]), "=f"(f[3]) : "r"(w), "r"(kHalf | (kHalf << 16)));
+        : "=f"(f[0]), "=f"(f[1]), "=f"(f[2]), "=f"(f[3]) : "r"(a), "r"(b), "r"(kHalf | (kHalf << 16)));
 }
 
 // four E4M3 codes (one word) -> four 6-bit codes, one per byte
@@ -617,6 +625,59 @@ __device__ __forceinline__ uint32_t ss_e4m3_word_soft(uint32_t x)
     return m | ((x >> sh) & (k01 << (FL::bits - 1)));
 }
 
+// Every legal pair, one element at a time (exact, slow): the reference path inside the kernels.
+template <class FH, class FL, int NWI, int NWO>
+__device__ __forceinline__ void ss_unit_by_element(const uint32_t (&in)[NWI], uint32_t (&out)[NWO])
+{
+#pragma unroll
+    for (int j = 0; j < NWO; ++j) out[j] = 0;
+    static_for<32>([&](auto i) {
+        constexpr int I = decltype(i)::value;
+        const uint32_t c = get_code<FH::bits, I>(in);
+        uint32_t d;
+        if constexpr (FH::kind == KIND_INT) d = ss_int_elem<FH, FL>(c);
+        else d = ss_fp_elem<FH, FL>(c);
+        put_code<FL::bits, I>(out, d);
+    });
+}
+
+template <class FH, class FL>
+__host__ __device__ constexpr bool ss_e4m3_has_fast_path()
+{
+    return FH::id == MXQ_FP8_E4M3 && FL::id != MXQ_FP8_E4M3 &&
+           (FL::hw_cvt || FL::id == MXQ_FP7_E3M3 || FL::id == MXQ_FP5_E2M2);
+}
+
+__device__ __forceinline__ bool unit_has_e4m3_nan(const uint32_t (&in)[8])
+{
+    bool nan = false;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) nan |= has_e4m3_nan(in[j]);
+    return nan;
+}
+
+// The 32 E4M3 codes of one lane, none of them a NaN code, to any lower MXFP format.
+template <class FL, int NWO>
+__device__ __forceinline__ void ss_e4m3_unit_fast(const uint32_t (&in)[8], uint32_t (&out)[NWO])
+{
+    if constexpr (FL::hw_cvt && FL::bits == 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[j] = ss_e4m3_words_to_e2m1(in[2 * j], in[2 * j + 1]);
+    } else if constexpr (FL::hw_cvt) {
+        uint32_t z[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) z[j] = squeeze6(ss_e4m3_word_to6<FL>(in[j]));
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+            join24(z[4 * g + 0], z[4 * g + 1], z[4 * g + 2], z[4 * g + 3], out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
+    } else {
+        uint32_t z[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) z[j] = ss_e4m3_word_soft<FL>(in[j]);
+        pack_code_bytes<FL::bits>(z, out);
+    }
+}
+
 // Convert the 32 codes of one lane.  in: 8*FH::bits/8... words of the high format's bitstream.
 template <class FH, class FL, int NWI, int NWO>
 __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint32_t (&out)[NWO])
@@ -646,58 +707,11 @@ __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint
 #pragma unroll
         for (int j = 0; j < 8; ++j) z[j] = ss_int8_word<FL::bits>(in[j]);
         pack_code_bytes<FL::bits>(z, out);
-    } else if constexpr (FH::id == MXQ_FP8_E4M3 && FL::hw_cvt) {
-        bool nan = false;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) nan |= has_e4m3_nan(in[j]);
-        if (!nan) {
-            if constexpr (FL::bits == 4) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) out[j] = ss_e4m3_words_to_e2m1(in[2 * j], in[2 * j + 1]);
-            } else {
-                uint32_t z[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) z[j] = squeeze6(ss_e4m3_word_to6<FL>(in[j]));
-#pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    join24(z[4 * g + 0], z[4 * g + 1], z[4 * g + 2], z[4 * g + 3], out[3 * g + 0], out[3 * g + 1],
-                           out[3 * g + 2]);
-                }
-            }
-        } else {
-            // an E4M3 NaN code (never produced by the quantizer): exact scalar path
-#pragma unroll
-            for (int j = 0; j < NWO; ++j) out[j] = 0;
-            static_for<32>([&](auto i) {
-                constexpr int I = decltype(i)::value;
-                put_code<FL::bits, I>(out, ss_fp_elem<FH, FL>(get_code<FH::bits, I>(in)));
-            });
-        }
-    } else if constexpr (FH::id == MXQ_FP8_E4M3 && (FL::id == MXQ_FP7_E3M3 || FL::id == MXQ_FP5_E2M2)) {
-        bool nan = false;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) nan |= has_e4m3_nan(in[j]);
-        if (!nan) {
-            uint32_t z[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) z[j] = ss_e4m3_word_soft<FL>(in[j]);
-            pack_code_bytes<FL::bits>(z, out);
-        } else {
-            static_for<32>([&](auto i) {
-                constexpr int I = decltype(i)::value;
-                put_code<FL::bits, I>(out, ss_fp_elem<FH, FL>(get_code<FH::bits, I>(in)));
-            });
-        }
+    } else if constexpr (ss_e4m3_has_fast_path<FH, FL>()) {
+        if (!unit_has_e4m3_nan(in)) ss_e4m3_unit_fast<FL>(in, out);
+        else ss_unit_by_element<FH, FL>(in, out);     // an E4M3 NaN code (never produced by the quantizer)
     } else {
-        // every other pair (including non-anchor sources): element by element
-        static_for<32>([&](auto i) {
-            constexpr int I = decltype(i)::value;
-            uint32_t c = get_code<FH::bits, I>(in);
-            uint32_t d;
-            if constexpr (FH::kind == KIND_INT) d = ss_int_elem<FH, FL>(c);
-            else d = ss_fp_elem<FH, FL>(c);
-            put_code<FL::bits, I>(out, d);
-        });
+        ss_unit_by_element<FH, FL>(in, out);          // every other pair, including non-anchor sources
     }
 }
 
@@ -826,10 +840,22 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
             out_scales2[unit] = ss_scale_byte(sb[u], de2);
         }
         uint32_t o1[OB1 / 4], o2[OB2 / 4];
-        slice_scale_unit<FH, FL1>(w[u], o1);
+        if constexpr (ss_e4m3_has_fast_path<FH, FL1>() && ss_e4m3_has_fast_path<FH, FL2>()) {
+            // one NaN-code check, both conversions in one straight line: what they share (the widening
+            // of the anchor codes, the scaled values when de is the same) is computed once
+            if (!unit_has_e4m3_nan(w[u])) {
+                ss_e4m3_unit_fast<FL1>(w[u], o1);
+                ss_e4m3_unit_fast<FL2>(w[u], o2);
+            } else {
+                ss_unit_by_element<FH, FL1>(w[u], o1);
+                ss_unit_by_element<FH, FL2>(w[u], o2);
+            }
+        } else {
+            slice_scale_unit<FH, FL1>(w[u], o1);
+            slice_scale_unit<FH, FL2>(w[u], o2);
+        }
         if constexpr (StagedTile<OB1>::use) store_bytes<OB1>(stage1 + (u * 32 + (threadIdx.x & 31)) * OB1, o1);
         else if (unit < nunits) store_bytes<OB1>(out_codes1 + unit * OB1, o1);
-        slice_scale_unit<FH, FL2>(w[u], o2);
         if constexpr (StagedTile<OB2>::use) store_bytes<OB2>(stage2 + (u * 32 + (threadIdx.x & 31)) * OB2, o2);
         else if (unit < nunits) store_bytes<OB2>(out_codes2 + unit * OB2, o2);
     }
