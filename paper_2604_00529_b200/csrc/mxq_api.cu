@@ -1,6 +1,5 @@
 // The C ABI of libmxq (declared in include/mxq.h): argument validation on the host, then the
 // per-operation launchers.  Nothing here synchronises the device.
-#include <cstring>
 #include <mutex>
 #include <vector>
 

@@ -7,7 +7,8 @@
 //   quantize / fake_quant : unit = 32 B of FP32/BF16 input (8 / 16 elements); a block of 32
 //                           elements spans 4 / 2 adjacent lanes, whose maxima meet by xor-shuffles.
 //   slice_scale           : unit = 32 element codes = one block per lane, no cross-lane traffic.
-//   dequantize            : unit = 32 element codes in, 64 / 128 B out.
+//   dequantize            : to 16-bit outputs a unit is 32 element codes (64 B out); to FP32 it is 32 B
+//                           of output (8 elements), see dequantize_wide_kernel.
 //
 // All of them are bound by HBM traffic, with the integer/logic pipe (64 lanes per clock per SM) as
 // the second bound; the arithmetic below is shaped to stay under it: packed 16-bit maxima, round-down
