@@ -165,6 +165,25 @@ size_t mxq_tiled_scales_bytes(size_t rows, size_t kblocks);
 int mxq_tile_scales(const uint8_t *scales, size_t rows, size_t kblocks, uint8_t *tiled, mxq_stream stream);
 
 /*
+ * Q_f (Eq. 1-3) and Slice-and-Scale (Eq. 5) of a row-major [rows, cols] matrix with the scale bytes
+ * written directly in the tiled order above, by the producing kernel: the same bytes as
+ * mxq_quantize / mxq_slice_scale followed by mxq_tile_scales(rows, cols / 32), without the extra
+ * pass.  The element codes are the same plain packed streams.  MXFP formats only (the formats the
+ * block-scaled multiply takes; MXQ_ERR_FORMAT otherwise), block == 32 only (MXQ_ERR_BLOCK), cols a
+ * multiple of 32 and rows * cols / 32 below 2^32 (MXQ_ERR_SIZE).  When rows is not a multiple of 128
+ * or cols / 32 not a multiple of 4, the tiled buffer is first cleared on `stream`, so that the
+ * uncovered part of the edge tiles reads 0.
+ *   src / codes, scales   [in]  device, as for mxq_quantize / mxq_slice_scale (plain stored scales)
+ *   codes / out_codes     [out] device, mxq_codes_bytes(rows * cols, fmt) bytes, 32-byte aligned
+ *   tiled_scales          [out] device, mxq_tiled_scales_bytes(rows, cols / 32) bytes, 16-byte aligned
+ */
+int mxq_quantize_tiled(const void *src, int src_dtype, size_t rows, size_t cols, int fmt, int block,
+                       void *codes, uint8_t *tiled_scales, mxq_stream stream);
+int mxq_slice_scale_tiled(const void *codes, const uint8_t *scales, size_t rows, size_t cols, int block,
+                          int src_fmt, int dst_fmt, void *out_codes, uint8_t *out_tiled_scales,
+                          mxq_stream stream);
+
+/*
  * Fused fake-quant forward, Eq. 6 in reconstructed form; nothing but the result leaves
  * the SM.  mode MXQ_FQ_DIRECT: dst = dequantize(Q_fmt(src)).  mode MXQ_FQ_VIA_ANCHOR:
  * dst = dequantize(Q_{A->fmt}(Q_A(src))) with A = MXINT8 for MXINT targets and MXFP8 E4M3

@@ -8,6 +8,6 @@ the library is missing or the tensors are not CUDA tensors.
 from .binding import (  # noqa: F401
     BF16, F32, FORMATS, FQ_DIRECT, FQ_VIA_ANCHOR, MxqError, codes_bytes, dequantize, fake_quant, fake_quant_batched,
     make_fq_items,
-    fake_quant_bwd, format_bits, library_path, load_library, make_items, quantize, scales_bytes, slice_scale,
-    slice_scale_batched, slice_scale_batched_static, slice_scale_multi, tile_scales, tiled_scales_bytes, status_string, STATIC_BATCH_MAX,
+    fake_quant_bwd, fake_quant_ste, format_bits, library_path, load_library, make_items, quantize, scales_bytes, slice_scale,
+    slice_scale_batched, slice_scale_batched_static, slice_scale_multi, quantize_tiled, slice_scale_tiled, tile_scales, tiled_scales_bytes, status_string, STATIC_BATCH_MAX,
 )

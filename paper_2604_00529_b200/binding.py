@@ -78,6 +78,10 @@ def load_library() -> ctypes.CDLL:
     L.mxq_tiled_scales_bytes.restype = sz
     L.mxq_tile_scales.argtypes = [vp, sz, sz, vp, vp]
     L.mxq_tile_scales.restype = i
+    L.mxq_quantize_tiled.argtypes = [vp, i, sz, sz, i, i, vp, vp, vp]
+    L.mxq_quantize_tiled.restype = i
+    L.mxq_slice_scale_tiled.argtypes = [vp, vp, sz, sz, i, i, i, vp, vp, vp]
+    L.mxq_slice_scale_tiled.restype = i
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
     L.mxq_slice_scale_batched_static.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
@@ -211,6 +215,38 @@ def tile_scales(scales: torch.Tensor, rows: int, kblocks: int, tiled: Optional[t
     return tiled
 
 
+def quantize_tiled(src: torch.Tensor, fmt: str, block: int = 32, codes: Optional[torch.Tensor] = None,
+                   tiled_scales: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """mxq_quantize_tiled: a 2-D [rows, cols] tensor -> (packed codes, scale bytes in the 128 x 4 tiled order)."""
+    L = load_library()
+    if src.dim() != 2:
+        raise ValueError("quantize_tiled takes a [rows, cols] matrix")
+    rows, cols = src.shape
+    if codes is None:
+        codes = torch.empty(codes_bytes(rows * cols, fmt), dtype=torch.uint8, device=src.device)
+    if tiled_scales is None:
+        tiled_scales = torch.empty(tiled_scales_bytes(rows, cols // 32), dtype=torch.uint8, device=src.device)
+    _check(L.mxq_quantize_tiled(_dev(src, "src"), _dtype_id(src), rows, cols, FORMATS[fmt], block, _dev(codes, "codes"),
+                                _dev(tiled_scales, "tiled_scales"), _stream(stream)), "mxq_quantize_tiled")
+    return codes, tiled_scales
+
+
+def slice_scale_tiled(codes: torch.Tensor, scales: torch.Tensor, rows: int, cols: int, src_fmt: str, dst_fmt: str,
+                      block: int = 32, out_codes: Optional[torch.Tensor] = None,
+                      out_tiled_scales: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """mxq_slice_scale_tiled: anchor codes + plain scales of a [rows, cols] matrix -> lower-format codes and
+    scale bytes in the 128 x 4 tiled order."""
+    L = load_library()
+    if out_codes is None:
+        out_codes = torch.empty(codes_bytes(rows * cols, dst_fmt), dtype=torch.uint8, device=codes.device)
+    if out_tiled_scales is None:
+        out_tiled_scales = torch.empty(tiled_scales_bytes(rows, cols // 32), dtype=torch.uint8, device=codes.device)
+    _check(L.mxq_slice_scale_tiled(_dev(codes, "codes"), _dev(scales, "scales"), rows, cols, block, FORMATS[src_fmt],
+                                   FORMATS[dst_fmt], _dev(out_codes, "out_codes"),
+                                   _dev(out_tiled_scales, "out_tiled_scales"), _stream(stream)), "mxq_slice_scale_tiled")
+    return out_codes, out_tiled_scales
+
+
 def fake_quant(src: torch.Tensor, fmt: str, block: int = 32, mode: int = FQ_DIRECT,
                dst: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """mxq_fake_quant: quantize-dequantize in one pass (dst may be src)."""
@@ -262,6 +298,29 @@ def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = Non
     _check(L.mxq_fake_quant_bwd(_dev(grad_out, "grad_out"), _dtype_id(grad_out), grad_out.numel(),
                                 _dev(grad_in, "grad_in"), _stream(stream)), "mxq_fake_quant_bwd")
     return grad_in
+
+
+class _FakeQuantSTE(torch.autograd.Function):
+    """Eq. 6 inside autograd: forward is mxq_fake_quant, backward the straight-through estimator."""
+
+    @staticmethod
+    def forward(ctx, x, fmt, block, mode, copy_grad):
+        ctx.copy_grad = copy_grad
+        return fake_quant(x.detach(), fmt, block, mode)
+
+    @staticmethod
+    def backward(ctx, grad_out):
+        # identity: the incoming gradient itself, or a copy of it made by mxq_fake_quant_bwd
+        g = fake_quant_bwd(grad_out.contiguous()) if ctx.copy_grad else grad_out
+        return g, None, None, None, None
+
+
+def fake_quant_ste(x: torch.Tensor, fmt: str, block: int = 32, mode: int = FQ_VIA_ANCHOR,
+                   copy_grad: bool = False) -> torch.Tensor:
+    """W_t of Eq. 6 as a differentiable function of W: the value is ``fake_quant(x, fmt, block, mode)``,
+    the gradient passes straight through (``copy_grad`` hands autograd a fresh copy instead of the
+    incoming tensor)."""
+    return _FakeQuantSTE.apply(x, fmt, block, mode, copy_grad)
 
 
 class ItemTable:

@@ -33,6 +33,50 @@ __device__ __forceinline__ void static_for(Fn&& fn)
 }
 
 // ------------------------------------------------------------------------------------------
+// Where a block's scale byte goes
+// ------------------------------------------------------------------------------------------
+// The kernels that produce scale bytes write them through put_scale(), overloaded on the type of
+// the destination: a plain pointer (byte of block i at scales[i], the library's stored form), or a
+// TiledScales record, which places them in the 128-row x 4-column tiles a block-scaled tensor-core
+// matrix multiply reads (the step that consumes W_t, Sec. 3.5): tile (r / 128, c / 4) is 512
+// consecutive bytes and holds the byte of row r, block-column c at
+// (r mod 32) * 16 + (r div 32 mod 4) * 4 + c mod 4.
+
+__device__ __forceinline__ void put_scale(uint8_t* scales, size_t blk, uint32_t byte)
+{
+    scales[blk] = (uint8_t)byte;
+}
+
+// Division of a 32-bit block index by the row length in blocks, by multiply and shift (the
+// round-up method for an invariant divisor: with s = ceil(log2 d) and m = floor(2^32 (2^s - d) / d) + 1,
+// n / d = (t + ((n - t) >> min(s, 1))) >> max(s - 1, 0) where t is the high word of m * n).  The host
+// fills in m and the two shifts (see make_tiled_scales in mxq_launch.h).
+struct TiledScales {
+    uint8_t* base;
+    uint32_t kblocks;      // block-columns per row (the divisor)
+    uint32_t magic, shift1, shift2;
+    uint32_t col_tiles;    // ceil(kblocks / 4)
+};
+
+inline TiledScales make_tiled_scales(uint8_t* base, uint32_t kblocks)      // 1 <= kblocks <= 2^31
+{
+    uint32_t s = 0;
+    while ((1ull << s) < kblocks) ++s;
+    const uint64_t m = ((1ull << 32) * ((1ull << s) - kblocks)) / kblocks + 1;
+    return TiledScales{base, kblocks, (uint32_t)m, s < 1 ? s : 1u, s > 1 ? s - 1 : 0u, (kblocks + 3) / 4};
+}
+
+__device__ __forceinline__ void put_scale(const TiledScales& t, size_t blk, uint32_t byte)
+{
+    const uint32_t n = (uint32_t)blk;
+    const uint32_t hi = __umulhi(t.magic, n);
+    const uint32_t r = (hi + ((n - hi) >> t.shift1)) >> t.shift2;
+    const uint32_t c = n - r * t.kblocks;
+    const size_t tile = (size_t)(r >> 7) * t.col_tiles + (c >> 2);
+    t.base[tile * 512 + (r & 31u) * 16u + ((r >> 5) & 3u) * 4u + (c & 3u)] = (uint8_t)byte;
+}
+
+// ------------------------------------------------------------------------------------------
 // Source element types
 // ------------------------------------------------------------------------------------------
 
@@ -246,10 +290,9 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
     }
 }
 
-template <class T, class F, int BLOCK, int U, int THREADS>
+template <class T, class F, int BLOCK, int U, int THREADS, class SCALES = uint8_t*>
 __global__ void __launch_bounds__(THREADS)
-quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes,
-                uint8_t* __restrict__ scales)
+quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes, SCALES scales)
 {
     pdl_release();
     constexpr int LPB = BLOCK / T::epl;                 // lanes per block
@@ -292,7 +335,7 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
             if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + lane) * OB, out);
             if (unit < nunits) {
                 if constexpr (!StagedTile<OB>::use) store_bytes<OB>(codes + unit * OB, out);
-                if (lane % LPB == 0) scales[unit / LPB] = (uint8_t)s.byte;
+                if (lane % LPB == 0) put_scale(scales, unit / LPB, s.byte);
             }
         }
         if constexpr (StagedTile<OB>::use) {
@@ -725,10 +768,10 @@ __device__ __forceinline__ uint8_t ss_scale_byte(uint32_t b, int de)
 // One warp tile (32 U lane units) of one tensor; shared by the single-tensor and the batched
 // kernels.  The scale bytes are an element-wise stream of their own: lane unit i also converts
 // scale i, and scale nunits + i when the block is smaller than a lane unit (block 16).
-template <class FH, class FL, int U>
+template <class FH, class FL, int U, class SCALES>
 __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
                                                  size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes,
-                                                 uint8_t* __restrict__ out_scales, size_t tile, uint8_t* stage)
+                                                 const SCALES& out_scales, size_t tile, uint8_t* stage)
 {
     constexpr int IB = 4 * FH::bits, OB = 4 * FL::bits;      // bytes per lane unit
     constexpr int NWI = IB / 4, NWO = OB / 4;
@@ -749,7 +792,7 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t unit = u0 + u * 32;
-        if (unit < nscales) out_scales[unit] = ss_scale_byte(sb[u], de);
+        if (unit < nscales) put_scale(out_scales, unit, ss_scale_byte(sb[u], de));
         uint32_t out[NWO];
         slice_scale_unit<FH, FL>(w[u], out);
         if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + (threadIdx.x & 31)) * OB, out);
@@ -763,7 +806,7 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const size_t i = nunits + u0 + u * 32;
-            if (i < nscales) out_scales[i] = ss_scale_byte(scales[i], de);
+            if (i < nscales) put_scale(out_scales, i, ss_scale_byte(scales[i], de));
         }
     }
 }
@@ -782,10 +825,10 @@ __device__ __forceinline__ uint8_t* slice_scale_stage()
     }
 }
 
-template <class FH, class FL, int U, int THREADS>
+template <class FH, class FL, int U, int THREADS, class SCALES = uint8_t*>
 __global__ void __launch_bounds__(THREADS)
 slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
-                   size_t nscales, uint8_t* __restrict__ out_codes, uint8_t* __restrict__ out_scales)
+                   size_t nscales, uint8_t* __restrict__ out_codes, SCALES out_scales)
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);

@@ -30,6 +30,12 @@ int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int b
 int launch_slice_scale2(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt1,
                         int dst_fmt2, void* out_codes1, uint8_t* out_scales1, void* out_codes2, uint8_t* out_scales2,
                         cudaStream_t stream);
+// The same two operations with the scale bytes written in 128 x 4 tiles (block 32, kblocks block-columns
+// per row); the caller has zeroed the tiled buffer when the matrix leaves part of a tile uncovered.
+int launch_quantize_tiled(const void* src, int dtype, size_t n, int fmt, void* codes, uint8_t* tiled,
+                          uint32_t kblocks, cudaStream_t stream);
+int launch_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t n, int src_fmt, int dst_fmt,
+                             void* out_codes, uint8_t* out_tiled, uint32_t kblocks, cudaStream_t stream);
 int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
                       cudaStream_t stream);
 // Fused fake-quant over up to kFqBatchItemsMax tensors in one launch; `items_host` is a HOST array

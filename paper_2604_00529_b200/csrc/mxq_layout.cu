@@ -3,7 +3,12 @@
 // E8M0 bytes is cut into tiles of 128 rows x 4 block-columns; a tile is 512 consecutive bytes, and
 // inside it the byte of row r, column c sits at (r mod 32) * 16 + (r div 32) * 4 + c.  Tiles follow
 // one another row-tile by row-tile.  Rows and columns beyond the matrix are filled with byte 0.
+//
+// mxq_tile_scales re-orders stored scale bytes in a pass of its own; mxq_quantize_tiled and
+// mxq_slice_scale_tiled are Q_f and Slice-and-Scale with the scale bytes written in that order by the
+// producing kernel itself (put_scale in mxq_kernels.cuh), which saves the pass.
 #include "mxq_access.cuh"
+#include "mxq_codec.cuh"
 #include "mxq_launch.h"
 
 namespace mxq {
@@ -70,6 +75,67 @@ int mxq_tile_scales(const uint8_t* scales, size_t rows, size_t kblocks, uint8_t*
     if (kblocks % 4 == 0)
         return launch_kernel(tile_scales_kernel<true>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
     return launch_kernel(tile_scales_kernel<false>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
+}
+
+namespace {
+
+// Checks shared by the two fused entry points.  On MXQ_OK with *n == 0 there is nothing to do.
+int check_tiled(size_t rows, size_t cols, int block, size_t* n, uint32_t* kblocks)
+{
+    *n = 0;
+    if (block != 32) return MXQ_ERR_BLOCK;                 // the tiled order is defined for 32-element blocks
+    if (cols % 32) return MXQ_ERR_SIZE;
+    if (rows == 0 || cols == 0) return MXQ_OK;
+    const size_t kb = cols / 32;
+    if (kb > ((size_t)1 << 31) || rows > (((size_t)1 << 32) - 1) / kb) return MXQ_ERR_SIZE;   // block index in 32 bits
+    *n = rows * cols;
+    *kblocks = (uint32_t)kb;
+    return MXQ_OK;
+}
+
+// Tiles that the matrix covers only in part keep byte 0 where no block lands: clear the buffer first.
+int clear_partial_tiles(uint8_t* tiled, size_t rows, size_t kblocks, cudaStream_t s)
+{
+    if (rows % 128 == 0 && kblocks % 4 == 0) return MXQ_OK;
+    if (cudaMemsetAsync(tiled, 0, mxq_tiled_scales_bytes(rows, kblocks), s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    return MXQ_OK;
+}
+
+}  // namespace
+
+int mxq_quantize_tiled(const void* src, int src_dtype, size_t rows, size_t cols, int fmt, int block, void* codes,
+                       uint8_t* tiled_scales, mxq_stream stream)
+{
+    if (fmt_info(fmt).kind != KIND_FP || (src_dtype != MXQ_F32 && src_dtype != MXQ_BF16)) return MXQ_ERR_FORMAT;
+    size_t n;
+    uint32_t kblocks = 0;
+    if (int rc = check_tiled(rows, cols, block, &n, &kblocks)) return rc;
+    if (n == 0) return MXQ_OK;
+    if (!src || !codes || !tiled_scales) return MXQ_ERR_NULL;
+    if (!aligned(src, 32) || !aligned(codes, 32) || !aligned(tiled_scales, 16)) return MXQ_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = clear_partial_tiles(tiled_scales, rows, kblocks, s)) return rc;
+    return launch_quantize_tiled(src, src_dtype, n, fmt, codes, tiled_scales, kblocks, s);
+}
+
+int mxq_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t rows, size_t cols, int block, int src_fmt,
+                          int dst_fmt, void* out_codes, uint8_t* out_tiled_scales, mxq_stream stream)
+{
+    if (fmt_info(src_fmt).kind != KIND_FP || fmt_info(dst_fmt).kind != KIND_FP) return MXQ_ERR_FORMAT;
+    size_t n;
+    uint32_t kblocks = 0;
+    if (int rc = check_tiled(rows, cols, block, &n, &kblocks)) return rc;
+    if (!ss_pair_ok(src_fmt, dst_fmt)) return MXQ_ERR_PAIR;
+    if (n == 0) return MXQ_OK;
+    if (!codes || !scales || !out_codes || !out_tiled_scales) return MXQ_ERR_NULL;
+    if (!aligned(codes, 32) || !aligned(out_codes, 32) || !aligned(scales, 16) || !aligned(out_tiled_scales, 16))
+        return MXQ_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = clear_partial_tiles(out_tiled_scales, rows, kblocks, s)) return rc;
+    return launch_slice_scale_tiled(codes, scales, n, src_fmt, dst_fmt, out_codes, out_tiled_scales, kblocks, s);
 }
 
 }  // extern "C"

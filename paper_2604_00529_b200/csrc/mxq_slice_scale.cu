@@ -27,6 +27,21 @@ int run_single(const void* codes, const uint8_t* scales, size_t n, int block, vo
 }
 
 template <class FH, class FL>
+int run_single_tiled(const void* codes, const uint8_t* scales, size_t n, void* out_codes, const TiledScales& out_tiled,
+                     cudaStream_t stream)
+{
+    if constexpr (ss_pair_ok(FH::id, FL::id) && FL::kind == KIND_FP) {
+        auto kern = slice_scale_kernel<FH, FL, kU, kThreads, TiledScales>;
+        const size_t nunits = n / 32;
+        const size_t ntiles = (nunits + 32 * kU - 1) / (32 * kU);
+        return launch_kernel(kern, grid_for_tiles(ntiles, kThreads), kThreads, stream, static_cast<const uint8_t*>(codes),
+                             scales, nunits, nunits, static_cast<uint8_t*>(out_codes), out_tiled);
+    } else {
+        return MXQ_ERR_PAIR;
+    }
+}
+
+template <class FH, class FL>
 int run_table(const SsDeviceItem* items_dev, int count, size_t total_tiles, cudaStream_t stream)
 {
     if constexpr (ss_pair_ok(FH::id, FL::id)) {
@@ -65,6 +80,16 @@ int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int b
 {
     MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
         MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_single<FH, FL>(codes, scales, n, block, out_codes, out_scales, stream); });
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+int launch_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t n, int src_fmt, int dst_fmt,
+                             void* out_codes, uint8_t* out_tiled, uint32_t kblocks, cudaStream_t stream)
+{
+    const TiledScales sink = make_tiled_scales(out_tiled, kblocks);
+    MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_single_tiled<FH, FL>(codes, scales, n, out_codes, sink, stream); });
     });
     return MXQ_ERR_FORMAT;
 }

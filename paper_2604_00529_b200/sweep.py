@@ -1,6 +1,6 @@
 """Bandwidth sweep of libmxq on one GPU.
 
-    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--all-formats] [--graph] [--json out.json]
+    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--all-formats] [--tiled] [--graph] [--json out.json]
 
 `--graph` times CUDA-graph replays instead of direct launches.  For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
 for every anchor-to-lower pair, reconstruction and the fused fake-quant, timed with CUDA events over
@@ -168,6 +168,35 @@ def all_formats(n: int, reps: int = 20):
     return out
 
 
+def tiled_scales(rows: int = 8192, cols: int = 8192, reps: int = 50):
+    """Scale bytes in the tiled order of a block-scaled matmul: the producing kernel writing them
+    itself (quantize_tiled, slice_scale_tiled) against the plain kernel followed by tile_scales."""
+    n = rows * cols
+    g = torch.Generator(device="cuda").manual_seed(2)
+    copies = 4
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    x = [(torch.randn(rows, cols, device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(copies)]
+    anchor = [mxq.quantize(x[j], "e4m3", BLOCK) for j in range(copies)]
+    oc = [torch.empty(n, **u8) for _ in range(copies)]
+    plain = [torch.empty(n // BLOCK, **u8) for _ in range(copies)]
+    tiled = [torch.empty(mxq.tiled_scales_bytes(rows, cols // BLOCK), **u8) for _ in range(copies)]
+    out = {}
+    for fmt in ("e4m3", "e2m1"):
+        out["quantize_bf16_" + fmt] = {
+            "plain_us": _time(lambda j: mxq.quantize(x[j], fmt, BLOCK, oc[j], plain[j]), copies, reps),
+            "plain_then_tile_us": _time(lambda j: (mxq.quantize(x[j], fmt, BLOCK, oc[j], plain[j]),
+                                                   mxq.tile_scales(plain[j], rows, cols // BLOCK, tiled[j])), copies, reps),
+            "fused_us": _time(lambda j: mxq.quantize_tiled(x[j], fmt, BLOCK, oc[j], tiled[j]), copies, reps)}
+    for dst in ("e2m3", "e2m1"):
+        out["slice_scale_e4m3_" + dst] = {
+            "plain_us": _time(lambda j: mxq.slice_scale(*anchor[j], n, "e4m3", dst, BLOCK, oc[j], plain[j]), copies, reps),
+            "plain_then_tile_us": _time(lambda j: (mxq.slice_scale(*anchor[j], n, "e4m3", dst, BLOCK, oc[j], plain[j]),
+                                                   mxq.tile_scales(plain[j], rows, cols // BLOCK, tiled[j])), copies, reps),
+            "fused_us": _time(lambda j: mxq.slice_scale_tiled(*anchor[j], rows, cols, "e4m3", dst, BLOCK, oc[j], tiled[j]),
+                              copies, reps)}
+    return {k: {a: round(b, 2) for a, b in v.items()} for k, v in out.items()}
+
+
 def whole_model(reps: int = 5):
     """Anchor -> target for the 224 tensors of the 8B Llama-shaped set, one batched launch per target.
     Anchors hold seeded random codes (the conversion's speed does not depend on the values)."""
@@ -219,6 +248,7 @@ def main():
     ap.add_argument("--max-log2", type=int, default=31)
     ap.add_argument("--model", action="store_true")
     ap.add_argument("--all-formats", action="store_true", help="every element format of the paper at 2^26 elements")
+    ap.add_argument("--tiled", action="store_true", help="tiled scale order at 8192 x 8192: fused against two passes")
     ap.add_argument("--json", default=None)
     ap.add_argument("--graph", action="store_true",
                     help="capture each timed loop in a CUDA graph and time its replay: the figures then exclude the "
@@ -251,6 +281,12 @@ def main():
         print("all formats, 2^26 elements: GB/s (us)")
         for f, row in fm.items():
             print("  %-5s " % f + "  ".join("%s %6.0f (%5.1f)" % (op, g, us) for op, (us, g) in row.items()))
+    if args.tiled:
+        result["tiled"] = tiled_scales()
+        print("scales in the tiled order, BF16 8192 x 8192: us per call")
+        for name, r in result["tiled"].items():
+            print("  %-24s plain %6.2f | plain then tile_scales %6.2f | fused %6.2f" %
+                  (name, r["plain_us"], r["plain_then_tile_us"], r["fused_us"]))
     if args.model:
         result["model"] = whole_model()
         for name, r in result["model"].items():

@@ -81,6 +81,23 @@ def test_argument_checks_answer_on_the_host(L):
     assert ts(A + 4, 128, 4, A, None) == E_ALIGN and ts(A, 128, 4, A + 8, None) == E_ALIGN
     assert L.mxq_tiled_scales_bytes(1, 1) == 512 and L.mxq_tiled_scales_bytes(129, 5) == 2 * 2 * 512
     assert L.mxq_tiled_scales_bytes(8192, 256) == 8192 * 256
+    qt = L.mxq_quantize_tiled                       # (src, dtype, rows, cols, fmt, block, codes, tiled, stream)
+    assert qt(None, 1, 0, 64, F["e4m3"], 32, None, None, None) == OK
+    assert qt(A, 1, 2, 64, F["int8"], 32, A, A, None) == E_FORMAT            # MXFP formats only
+    assert qt(A, 7, 2, 64, F["e4m3"], 32, A, A, None) == E_FORMAT
+    assert qt(A, 1, 2, 64, F["e4m3"], 64, A, A, None) == E_BLOCK             # tiles are defined for block 32
+    assert qt(A, 1, 2, 48, F["e4m3"], 32, A, A, None) == E_SIZE
+    assert qt(A, 1, 1 << 31, 64, F["e4m3"], 32, A, A, None) == E_SIZE        # 2^32 blocks
+    assert qt(A, 1, 2, 64, F["e4m3"], 32, A, None, None) == E_NULL
+    assert qt(A, 1, 2, 64, F["e4m3"], 32, A, A + 8, None) == E_ALIGN
+    st = L.mxq_slice_scale_tiled                    # (codes, scales, rows, cols, block, src, dst, out_codes, out_tiled, stream)
+    assert st(None, None, 4, 0, 32, F["e4m3"], F["e2m1"], None, None, None) == OK
+    assert st(A, A, 2, 64, 32, F["int8"], F["int4"], A, A, None) == E_FORMAT
+    assert st(A, A, 2, 64, 32, F["e2m1"], F["e4m3"], A, A, None) == E_PAIR
+    assert st(A, A, 2, 64, 16, F["e4m3"], F["e2m1"], A, A, None) == E_BLOCK
+    assert st(A, A, 2, 80, 32, F["e4m3"], F["e2m1"], A, A, None) == E_SIZE
+    assert st(A, None, 2, 64, 32, F["e4m3"], F["e2m1"], A, A, None) == E_NULL
+    assert st(A, A, 2, 64, 32, F["e4m3"], F["e2m1"], A + 16, A, None) == E_ALIGN
     dq = L.mxq_dequantize
     assert dq(A, A, 64, F["int4"], 32, A, 5, None) == E_FORMAT
     assert dq(A, None, 64, F["int4"], 32, A, 0, None) == E_NULL

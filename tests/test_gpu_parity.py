@@ -330,6 +330,20 @@ def test_fake_quant_in_place_and_backward():
     assert torch.equal(mxq.fake_quant_bwd(g32), g32)
 
 
+@pytest.mark.parametrize("copy_grad", [False, True])
+def test_fake_quant_inside_autograd_is_straight_through(copy_grad):
+    """Eq. 6 as a differentiable function: value = the oracle's fake-quant, dL/dW = dL/dW_t bit for bit."""
+    w_bits = inputs.to_bf16_bits(_mixed_f32(257, 11))
+    w = to_dev(w_bits).view(257, 32).requires_grad_(True)
+    wt = mxq.fake_quant_ste(w, "e2m1", 32, mxq.FQ_VIA_ANCHOR, copy_grad=copy_grad)
+    assert bits_equal(to_host(wt.detach().reshape(-1)), orc.fake_quant(w_bits, "e2m1", mode=orc.FQ_VIA_ANCHOR))
+    up = to_dev(inputs.to_bf16_bits(np.random.default_rng(3).standard_normal(w_bits.size).astype(np.float32))).view(257, 32)
+    wt.backward(up)
+    torch.cuda.synchronize()
+    assert torch.equal(w.grad.view(torch.int16), up.view(torch.int16))
+    assert (w.grad.data_ptr() != up.data_ptr()) or not copy_grad
+
+
 @pytest.mark.parametrize("count", [1, 7, 512, 513, 1100])
 @pytest.mark.parametrize("bf16", [True, False])
 def test_fake_quant_batched_matches_oracle(count, bf16):

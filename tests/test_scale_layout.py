@@ -52,6 +52,82 @@ def test_gpu_tile_scales_matches_oracle(rows, kb):
     assert np.all(got[:256] == 0xA5) and np.all(got[256 + nbytes:] == 0xA5)
 
 
+_FP = ("e4m3", "e3m3", "e3m2", "e2m3", "e2m2", "e2m1")
+# row counts and row lengths (in blocks) that leave whole tiles, ragged tiles in either direction, rows
+# shorter than a warp tile (so that one warp's blocks span several rows) and a non-power-of-two divisor
+_SHAPES = [(1, 1), (3, 2), (128, 4), (129, 4), (128, 5), (300, 7), (257, 3), (1000, 33), (512, 128), (96, 448)]
+
+
+def _bf16_matrix(rows, cols, seed):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((rows, cols)) * 2.0 ** rng.integers(-20, 21, (rows, cols // 32)).repeat(32, axis=1)
+    return inputs.to_bf16_bits(x.astype(np.float32).reshape(-1))
+
+
+def _guarded(nbytes):
+    return torch.full((nbytes + 512,), 0xA5, dtype=torch.uint8, device="cuda")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows,kb", _SHAPES)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_gpu_quantize_tiled_equals_quantize_then_tile(rows, kb, dtype):
+    """Fused entry point against the oracle's quantizer followed by the oracle's tiling, every MXFP format."""
+    cols = kb * 32
+    bits = _bf16_matrix(rows, cols, rows * 7 + kb)
+    if dtype == "bf16":
+        host = bits
+        x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16).view(rows, cols)
+    else:
+        host = (bits.astype(np.uint32) << 16).view(np.float32)
+        x = torch.from_numpy(host).cuda().view(rows, cols)
+    nbytes = mxq.tiled_scales_bytes(rows, kb)
+    for fmt in _FP:
+        wc, ws = orc.quantize(host, fmt, 32)
+        buf = _guarded(nbytes)
+        codes, _ = mxq.quantize_tiled(x, fmt, 32, tiled_scales=buf[256:256 + nbytes])
+        torch.cuda.synchronize()
+        got = buf.cpu().numpy()
+        assert np.array_equal(got[256:256 + nbytes], orc.tile_scales(ws.reshape(rows, kb), rows, kb)), fmt
+        assert np.all(got[:256] == 0xA5) and np.all(got[256 + nbytes:] == 0xA5)
+        assert np.array_equal(codes.cpu().numpy(), orc.pack(wc, orc.bits(fmt))), fmt
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows,kb", _SHAPES)
+def test_gpu_slice_scale_tiled_equals_slice_scale_then_tile(rows, kb):
+    cols = kb * 32
+    bits = _bf16_matrix(rows, cols, rows * 11 + kb)
+    ac, as_ = orc.quantize(bits, "e4m3", 32)
+    dc = torch.from_numpy(orc.pack(ac, 8)).cuda()
+    ds = torch.from_numpy(as_).cuda()
+    nbytes = mxq.tiled_scales_bytes(rows, kb)
+    for dst in _FP:
+        wc, ws = orc.slice_scale(ac, as_, "e4m3", dst, 32)
+        buf = _guarded(nbytes)
+        codes, _ = mxq.slice_scale_tiled(dc, ds, rows, cols, "e4m3", dst, 32, out_tiled_scales=buf[256:256 + nbytes])
+        torch.cuda.synchronize()
+        got = buf.cpu().numpy()
+        assert np.array_equal(got[256:256 + nbytes], orc.tile_scales(ws.reshape(rows, kb), rows, kb)), dst
+        assert np.all(got[:256] == 0xA5) and np.all(got[256 + nbytes:] == 0xA5)
+        assert np.array_equal(codes.cpu().numpy(), orc.pack(wc, orc.bits(dst))), dst
+
+
+@pytest.mark.gpu
+def test_gpu_tiled_entry_points_full_size_workload():
+    """BF16 8192 x 8192 (the bench's workload): fused outputs equal the two-pass outputs byte for byte
+    (the two-pass path is compared with the oracle at this size elsewhere)."""
+    x = torch.from_numpy(inputs.weight_bf16_student_t(8192, 8192, seed=1).view(np.int16)).cuda().view(torch.bfloat16)
+    x = x.view(8192, 8192)
+    codes, scales = mxq.quantize(x, "e4m3", 32)
+    tc, ts = mxq.quantize_tiled(x, "e4m3", 32)
+    assert torch.equal(tc, codes) and torch.equal(ts, mxq.tile_scales(scales, 8192, 256))
+    for dst in ("e2m3", "e2m1"):
+        lc, ls = mxq.slice_scale(codes, scales, x.numel(), "e4m3", dst, 32)
+        fc, fs = mxq.slice_scale_tiled(codes, scales, 8192, 8192, "e4m3", dst, 32)
+        assert torch.equal(fc, lc) and torch.equal(fs, mxq.tile_scales(ls, 8192, 256))
+
+
 def _mixed_matrix(rows, cols, seed):
     """Rows and 32-wide blocks at very different magnitudes, so that a misplaced scale is a gross error."""
     rng = np.random.default_rng(seed)
@@ -77,7 +153,10 @@ def test_block_scaled_matmul_consumes_codes_and_tiled_scales(fmt):
         x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
         codes, scales = mxq.quantize(x, fmt, 32)
         deq = mxq.dequantize(codes, scales, rows * K, fmt, 32, dtype=torch.float32).view(rows, K)
-        tiled = mxq.tile_scales(scales, rows, K // 32)
+        if name == "a":                              # one operand by the separate pass, the other by the fused kernel
+            tiled = mxq.tile_scales(scales, rows, K // 32)
+        else:
+            codes, tiled = mxq.quantize_tiled(x.view(rows, K), fmt, 32)
         qa[name] = (codes, tiled, deq)
     ref = qa["a"][2].double() @ qa["b"][2].double().t()
     if fmt == "e4m3":
