@@ -161,24 +161,26 @@ __device__ __forceinline__ uint32_t quantize_fp_hw_pair(float r0, float r1)
     return d;
 }
 
-// The two MXFP formats without a narrowing instruction, E3M3 and E2M2, have a hardware neighbour
-// with the same mantissa width and a wider exponent range (E4M3 and E3M2).  Where the target is a
-// normal number the neighbour's rounding is the target's rounding; below that the target's grid is
-// uniform (step 2^-5 / 2^-2) and rounding to it is one FP32 add of 2^18 / 2^21.
+// The two MXFP formats without a narrowing instruction, E3M3 and E2M2, are the hardware formats E4M3
+// and E3M2 with fewer binades: the mantissa width is the same, so 2^-k times the grid of E3M3 (E2M2),
+// k = the difference of the exponent biases (4 / 2), IS the grid of E4M3 (E3M2) up to the image of the
+// largest magnitude -- normal binades map to normal binades, and the uniform (subnormal) range of the
+// one lands exactly on the subnormal range of the other.  Hence code_F(r) = code_hw(r / 2^k), the
+// magnitude bits unchanged, except that the hardware format goes on above F's largest value: since
+// |r| < 2^(e_max + 1), the only code it can give beyond F's largest is the next one (a single bit,
+// 2^(bits - 1)), which is clipped back by subtracting that bit shifted down to 1.
 template <class F>
 struct SoftFp {
     static_assert(F::id == MXQ_FP7_E3M3 || F::id == MXQ_FP5_E2M2, "E3M3 or E2M2");
     static constexpr bool e3m3 = F::id == MXQ_FP7_E3M3;
     static constexpr int hw = e3m3 ? MXQ_FP8_E4M3 : MXQ_FP6_E3M2;        // the hardware neighbour
-    static constexpr uint32_t code_offset = e3m3 ? 32u : 8u;              // (bias_hw - bias_F) << mu
-    static constexpr uint32_t first_normal = e3m3 ? 40u : 12u;            // neighbour code of F's smallest normal
+    static constexpr int k = e3m3 ? 4 : 2;                                // bias_hw - bias_F
+    static constexpr float pre_scale = e3m3 ? 0.0625f : 0.25f;            // 2^-k
+    static constexpr float post_scale = e3m3 ? 16.0f : 4.0f;              // 2^k
     static constexpr uint32_t hw_mag_mask = e3m3 ? 0x7Fu : 0x1Fu;
-    static constexpr float grid_magic = e3m3 ? 262144.0f : 2097152.0f;    // 2^18 / 2^21: FP32 spacing = F's step
-    static constexpr float smallest_normal = e3m3 ? 0.25f : 1.0f;
-    static constexpr float largest = e3m3 ? 30.0f : 7.0f;
 };
 
-// Codes of four scaled elements (exact r = v / X, |r| < 2^(e_max + 1)), one per byte.
+// Codes of four elements given as r / 2^k (r = v / X exact, |r| < 2^(e_max + 1)), one per byte.
 template <class F>
 __device__ __forceinline__ uint32_t quantize_fp_soft_quad(float r0, float r1, float r2, float r3)
 {
@@ -191,33 +193,19 @@ __device__ __forceinline__ uint32_t quantize_fp_soft_quad(float r0, float r1, fl
     else
         asm("{ .reg .b16 l, h; cvt.rn.satfinite.e3m2x2.f32 l, %2, %1; cvt.rn.satfinite.e3m2x2.f32 h, %4, %3; mov.b32 %0, {l, h}; }"
             : "=r"(c) : "f"(r0), "f"(r1), "f"(r2), "f"(r3));
-    const uint32_t mag = c & (k01 * S::hw_mag_mask);
-    // normal regime: neighbour code - offset (the +128 keeps every byte's subtraction free of borrows),
-    // the one code above F's largest clipped back
-    uint32_t normal = (mag + k01 * (128u - S::code_offset)) & 0x7F7F7F7Fu;
-    normal -= (normal >> (F::bits - 1)) & k01;
-    // uniform regime: k = RNE(|r| / step) is the low byte of |r| + magic
-    const uint32_t s0 = __float_as_uint(fabsf(r0) + S::grid_magic), s1 = __float_as_uint(fabsf(r1) + S::grid_magic);
-    const uint32_t s2 = __float_as_uint(fabsf(r2) + S::grid_magic), s3 = __float_as_uint(fabsf(r3) + S::grid_magic);
-    const uint32_t k = __byte_perm(__byte_perm(s0, s1, 0x0040), __byte_perm(s2, s3, 0x0040), 0x5410);
-    uint32_t full;                                                        // 0xFF where the neighbour code is a normal of F
-    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(mag + k01 * (128u - S::first_normal)));
-    const uint32_t m = (normal & full) | (k & ~full);
+    uint32_t mag = c & (k01 * S::hw_mag_mask);
+    mag -= (mag >> (F::bits - 1)) & k01;                                  // the one code above F's largest
     // sign: top bit of the neighbour's code -> top bit of F's code (one position down in both cases)
-    return m | ((c >> 1) & (k01 << (F::bits - 1)));
+    return mag | ((c >> 1) & (k01 << (F::bits - 1)));
 }
 
-// The value (not the code) of one scaled element after quantization to E3M3 / E2M2; `n` is the element
-// rounded by the hardware neighbour (exact in FP32).
+// Two elements given as r / 2^k -> their two neighbour-format codes (code(r0) | code(r1) << 8), the
+// one code above F's largest clipped back: decoded as neighbour values they are P / 2^k.
 template <class F>
-__device__ __forceinline__ float quantize_fp_soft_value(float r, float n)
+__device__ __forceinline__ uint32_t quantize_fp_soft_pair(float r0, float r1)
 {
-    using S = SoftFp<F>;
-    const float a = fabsf(r);
-    const float uniform = (a + S::grid_magic) - S::grid_magic;            // RNE to the step, exact
-    const float normal = fminf(fabsf(n), S::largest);
-    const float m = a < S::smallest_normal ? uniform : normal;
-    return __uint_as_float(__float_as_uint(m) | (__float_as_uint(r) & 0x80000000u));
+    const uint32_t d = quantize_fp_hw_pair<Fmt<SoftFp<F>::hw>>(r0, r1);
+    return d - ((d >> (F::bits - 1)) & 0x0101u);
 }
 
 // Quantize two scaled-on-the-fly elements to an MXFP format; returns the two codes in the low `bits`

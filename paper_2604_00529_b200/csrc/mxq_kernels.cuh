@@ -266,10 +266,11 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
         // E3M3 / E2M2: four elements at a time through the hardware neighbour format
         constexpr int NQ = T::epl / 4;
         uint32_t z[NQ];
+        const float inv_k = inv * SoftFp<F>::pre_scale;          // exact: both are powers of two
         static_for<NQ>([&](auto qi) {
             constexpr int Q = decltype(qi)::value;
-            z[Q] = quantize_fp_soft_quad<F>(unit_elem<T, 4 * Q>(w) * inv, unit_elem<T, 4 * Q + 1>(w) * inv,
-                                            unit_elem<T, 4 * Q + 2>(w) * inv, unit_elem<T, 4 * Q + 3>(w) * inv);
+            z[Q] = quantize_fp_soft_quad<F>(unit_elem<T, 4 * Q>(w) * inv_k, unit_elem<T, 4 * Q + 1>(w) * inv_k,
+                                            unit_elem<T, 4 * Q + 2>(w) * inv_k, unit_elem<T, 4 * Q + 3>(w) * inv_k);
         });
         pack_code_bytes<F::bits>(z, out);
     } else {
@@ -405,24 +406,29 @@ __device__ __forceinline__ float2 fake_quant_pair(float v0, float v1, float inv)
         p.x = one(v0);
         p.y = one(v1);
     } else {
-        float r0 = v0 * inv, r1 = v1 * inv;
+        // E3M3 / E2M2 are quantized as 2^-k times the value in their hardware neighbour format (see SoftFp)
+        constexpr int k = [] { if constexpr (F::hw_cvt) return 0; else return SoftFp<F>::k; }();
+        float r0, r1;
         if constexpr (via) {
-            // anchor codes -> exact FP16 values -> divide by 2^de (exact) -> FP32
-            uint32_t a = quantize_fp_hw_pair<A>(r0, r1);
+            // anchor codes -> exact FP16 values -> divide by 2^(de + k) (exact) -> FP32
+            uint32_t a = quantize_fp_hw_pair<A>(v0 * inv, v1 * inv);
             uint32_t h2;
             asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)a));
-            constexpr uint32_t kHalf = (uint32_t)(15 - de) << 10;              // 2^-de as FP16
+            constexpr uint32_t kHalf = (uint32_t)(15 - de - k) << 10;          // 2^-(de + k) as FP16
             asm("mul.rn.f16x2 %0, %0, %1;" : "+r"(h2) : "r"(kHalf | (kHalf << 16)));
             asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h; }"
                 : "=f"(r0), "=f"(r1) : "r"(h2));
+        } else {
+            const float inv_k = inv * __uint_as_float((uint32_t)(127 - k) << 23);  // exact: powers of two
+            r0 = v0 * inv_k;
+            r1 = v1 * inv_k;
         }
         if constexpr (F::hw_cvt) {
             p = widen_hw_pair<F>(quantize_fp_hw_pair<F>(r0, r1));
         } else {
-            using N = Fmt<SoftFp<F>::hw>;
-            const float2 n = widen_hw_pair<N>(quantize_fp_hw_pair<N>(r0, r1));
-            p.x = quantize_fp_soft_value<F>(r0, n.x);
-            p.y = quantize_fp_soft_value<F>(r1, n.y);
+            p = widen_hw_pair<Fmt<SoftFp<F>::hw>>(quantize_fp_soft_pair<F>(r0, r1));
+            p.x *= SoftFp<F>::post_scale;
+            p.y *= SoftFp<F>::post_scale;
         }
     }
     return p;
@@ -626,47 +632,27 @@ __device__ __forceinline__ uint32_t ss_e4m3_words_to_e2m1(uint32_t w0, uint32_t 
 }
 
 // Eq. 5 for the two MXFP targets without a narrowing instruction, E3M3 (7 bits, de = 4) and E2M2
-// (5 bits, de = 6), on four E4M3 codes per register (no NaN codes among them).  Two facts do the work:
-//   - where the result is a normal number of the target, it follows from the anchor's magnitude
-//     code by integer arithmetic: E3M3 keeps the three mantissa bits (code - 64); E2M2 drops one
-//     (code / 2 rounded half to even, minus 48);
-//   - everywhere else the target's grid is uniform with step 2^-5 (E3M3) or 2^-2 (E2M2), and the
-//     magnitude code of k steps is k itself up to the second binade.  k = RNE(|v| / 16) for both, one
-//     FP16 fused multiply-add per pair of codes: |v| / 16 + C with C = 32 (step 2^-5... in units of
-//     the divided value) or 1024 (step 1) leaves k in the low mantissa bits of the sum.
-// The two regimes agree on the codes where they meet, so a per-byte threshold selects between them.
+// (5 bits, de = 6), on four E4M3 codes per register (no NaN codes among them): the anchor values
+// divided by 2^(de + k) = 2^8 (exact in FP16), converted to the hardware neighbour format whose grid is
+// 2^-k times the target's (see SoftFp), the one code above the target's largest clipped back.
 template <class FL>
 __device__ __forceinline__ uint32_t ss_e4m3_word_soft(uint32_t x)
 {
-    static_assert(FL::id == MXQ_FP7_E3M3 || FL::id == MXQ_FP5_E2M2, "E3M3 or E2M2");
-    constexpr bool e3m3 = FL::id == MXQ_FP7_E3M3;
+    using S = SoftFp<FL>;
     constexpr uint32_t k01 = 0x01010101u;
-    const uint32_t mag = x & 0x7F7F7F7Fu;
-    // k for the four codes: FP16 pairs, |v| * 2^-4 + C, low byte of each half
-    constexpr uint32_t kSixteenth = 0x2C002C00u;                        // 2^-4 as FP16 x2
-    constexpr uint32_t kC = e3m3 ? 0x50005000u : 0x64006400u;           // 32.0 / 1024.0 as FP16 x2
-    uint32_t a, b;
-    asm("{ .reg .b16 l, h;\n"
-        "  mov.b32 {l, h}, %2;\n"
-        "  cvt.rn.f16x2.e4m3x2 %0, l;  cvt.rn.f16x2.e4m3x2 %1, h;\n"
-        "  fma.rn.f16x2 %0, %0, %3, %4;  fma.rn.f16x2 %1, %1, %3, %4; }"
-        : "=r"(a), "=r"(b) : "r"(mag), "r"(kSixteenth), "r"(kC));
-    const uint32_t k = __byte_perm(a, b, 0x6420);
-    // the normal regime, valid from code kFrom on
-    constexpr uint32_t kFrom = e3m3 ? 72u : 104u;
-    uint32_t normal;
-    if constexpr (e3m3) {
-        normal = mag & 0x3F3F3F3Fu;                                      // code - 64 for codes >= 64
-    } else {
-        const uint32_t q = (mag >> 1) & 0x3F3F3F3Fu;
-        const uint32_t t = q + (mag & q & k01);                          // code / 2, ties to even: 52 .. 63
-        normal = t & 0x0F0F0F0Fu;                                        // - 48
-    }
-    uint32_t full;                                                       // 0xFF where code >= kFrom
-    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(mag + k01 * (128u - kFrom)));
-    const uint32_t m = (normal & full) | (k & ~full);
-    constexpr int sh = 8 - FL::bits;                                     // sign: bit 7 -> bit (bits - 1)
-    return m | ((x >> sh) & (k01 << (FL::bits - 1)));
+    constexpr int de = 8 - FL::emax;
+    uint32_t c;
+    float f[4];
+    e4m3_word_scaled<de + S::k>(x, f);
+    if constexpr (S::e3m3)
+        asm("{ .reg .b16 l, h; cvt.rn.satfinite.e4m3x2.f32 l, %2, %1; cvt.rn.satfinite.e4m3x2.f32 h, %4, %3; mov.b32 %0, {l, h}; }"
+            : "=r"(c) : "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]));
+    else
+        asm("{ .reg .b16 l, h; cvt.rn.satfinite.e3m2x2.f32 l, %2, %1; cvt.rn.satfinite.e3m2x2.f32 h, %4, %3; mov.b32 %0, {l, h}; }"
+            : "=r"(c) : "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]));
+    uint32_t mag = c & (k01 * S::hw_mag_mask);
+    mag -= (mag >> (FL::bits - 1)) & k01;
+    return mag | ((c >> 1) & (k01 << (FL::bits - 1)));
 }
 
 // Every legal pair, one element at a time (exact, slow): the reference path inside the kernels.
