@@ -239,6 +239,25 @@ int mxq_slice_scale_batched(const mxq_ss_item *items, int count, int block,
                             int src_fmt, int dst_fmt, mxq_stream stream);
 
 /*
+ * mxq_slice_scale_batched with every tensor's scale bytes written in the tiled order of
+ * mxq_tile_scales (the whole-model conversion of Sec. 3.5 handed straight to block-scaled matrix
+ * multiplies): item i is a row-major [rows, cols] matrix, and its results are those of
+ * mxq_slice_scale_tiled on it.  MXFP formats and block == 32 only, as there.  The items travel in
+ * the kernel's parameter space, 256 per launch (more items: more launches); nothing is allocated.
+ * Tiled buffers of matrices that do not cover whole tiles are cleared on `stream` first.
+ */
+typedef struct {
+    const void *codes;            /* [in]  device, anchor codes of rows * cols elements */
+    const uint8_t *scales;        /* [in]  device, rows * cols / 32 plain scale bytes */
+    size_t rows, cols;            /* cols a multiple of 32; rows * cols / 32 below 2^32 */
+    void *out_codes;              /* [out] device, mxq_codes_bytes(rows * cols, dst_fmt) bytes */
+    uint8_t *out_tiled_scales;    /* [out] device, mxq_tiled_scales_bytes(rows, cols / 32) bytes */
+} mxq_ss_tiled_item;
+
+int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item *items, int count, int block,
+                                  int src_fmt, int dst_fmt, mxq_stream stream);
+
+/*
  * The same conversion as mxq_slice_scale_batched for callers that cannot allocate device memory.
  * (The paper has no counterpart of this entry point; it exists for the library's users.)  Some
  * processes give all of HBM to a pool of their own at start-up, so a cudaMalloc made behind their

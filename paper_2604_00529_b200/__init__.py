@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     BF16, F32, FORMATS, FQ_DIRECT, FQ_VIA_ANCHOR, MxqError, codes_bytes, dequantize, fake_quant, fake_quant_batched,
     make_fq_items,
     fake_quant_bwd, fake_quant_ste, format_bits, library_path, load_library, make_items, quantize, scales_bytes, slice_scale,
-    slice_scale_batched, slice_scale_batched_static, slice_scale_multi, quantize_tiled, slice_scale_tiled, tile_scales, tiled_scales_bytes, status_string, STATIC_BATCH_MAX,
+    slice_scale_batched, slice_scale_batched_static, slice_scale_multi, quantize_tiled, slice_scale_tiled, slice_scale_tiled_batched, make_tiled_items, tile_scales, tiled_scales_bytes, status_string, STATIC_BATCH_MAX,
 )

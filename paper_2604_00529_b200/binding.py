@@ -39,6 +39,11 @@ class _Item(ctypes.Structure):
                 ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p)]
 
 
+class _TiledItem(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("rows", ctypes.c_size_t),
+                ("cols", ctypes.c_size_t), ("out_codes", ctypes.c_void_p), ("out_tiled_scales", ctypes.c_void_p)]
+
+
 _lib: Optional[ctypes.CDLL] = None
 
 
@@ -82,6 +87,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_quantize_tiled.restype = i
     L.mxq_slice_scale_tiled.argtypes = [vp, vp, sz, sz, i, i, i, vp, vp, vp]
     L.mxq_slice_scale_tiled.restype = i
+    L.mxq_slice_scale_tiled_batched.argtypes = [ctypes.POINTER(_TiledItem), i, i, i, i, vp]
+    L.mxq_slice_scale_tiled_batched.restype = i
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
     L.mxq_slice_scale_batched_static.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
@@ -349,6 +356,34 @@ def slice_scale_batched(items, src_fmt: str, dst_fmt: str, block: int = 32, stre
     table = items if isinstance(items, ItemTable) else ItemTable(items)
     _check(L.mxq_slice_scale_batched(table.array, len(table), block, FORMATS[src_fmt], FORMATS[dst_fmt],
                                      _stream(stream)), "mxq_slice_scale_batched")
+
+
+class TiledItemTable:
+    """A marshalled mxq_ss_tiled_item array (keeps the tensors alive), for buffers that persist."""
+
+    def __init__(self, items):
+        self.tensors = list(items)
+        self.array = (_TiledItem * len(self.tensors))()
+        for k, (c, s, rows, cols, oc, ot) in enumerate(self.tensors):
+            self.array[k] = _TiledItem(_dev(c, "codes"), _dev(s, "scales"), rows, cols, _dev(oc, "out_codes"),
+                                       _dev(ot, "out_tiled_scales"))
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_tiled_items(items) -> TiledItemTable:
+    """Marshal (codes, scales, rows, cols, out_codes, out_tiled_scales) tuples into an mxq_ss_tiled_item array."""
+    return TiledItemTable(items)
+
+
+def slice_scale_tiled_batched(items, src_fmt: str, dst_fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_slice_scale_tiled_batched over (codes, scales, rows, cols, out_codes, out_tiled_scales) tuples or a
+    TiledItemTable made from them."""
+    L = load_library()
+    table = items if isinstance(items, TiledItemTable) else TiledItemTable(items)
+    _check(L.mxq_slice_scale_tiled_batched(table.array, len(table), block, FORMATS[src_fmt], FORMATS[dst_fmt],
+                                           _stream(stream)), "mxq_slice_scale_tiled_batched")
 
 
 #: largest item count mxq_slice_scale_batched_static accepts (MXQ_STATIC_BATCH_MAX in include/mxq.h)

@@ -972,6 +972,43 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
                                 stage);
 }
 
+// The batched conversion with every tensor's scale bytes written in the tiled order (block 32): the
+// item carries the matrix's TiledScales record in place of a plain pointer.  K = 256 items of 72 bytes
+// ride in the kernel parameters.
+struct SsTiledDeviceItem {
+    const uint8_t* codes;
+    const uint8_t* scales;
+    uint8_t* out_codes;
+    TiledScales out_scales;
+    size_t nunits;
+    size_t tile_begin;
+};
+
+template <int K>
+struct SsTiledItemBlock {
+    SsTiledDeviceItem items[K];
+};
+
+template <class FH, class FL, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS)
+slice_scale_tiled_batched_kernel(const __grid_constant__ SsTiledItemBlock<K> blk, int count, size_t total_tiles)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
+    pdl_acquire();
+    if (tile >= total_tiles) return;
+    int lo = 0, hi = count - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (blk.items[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
+    }
+    const SsTiledDeviceItem& t = blk.items[lo];
+    slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nunits, t.out_codes, t.out_scales, tile - t.tile_begin,
+                                stage);
+}
+
 // ------------------------------------------------------------------------------------------
 // Reconstruction V^ = X P.  One lane = 32 codes.
 // ------------------------------------------------------------------------------------------

@@ -56,6 +56,12 @@ int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t 
 constexpr int kSsParamItemsMax = 512;
 int launch_slice_scale_batched_params(const SsDeviceItem* items_host, int count, size_t total_tiles, int src_fmt,
                                       int dst_fmt, cudaStream_t stream);
+// The batched launch with tiled scale outputs: up to kSsTiledItemsMax items (a HOST array, tile_begin
+// filled in) in the kernel's parameter space.
+struct SsTiledDeviceItem;
+constexpr int kSsTiledItemsMax = 256;
+int launch_slice_scale_tiled_batched(const SsTiledDeviceItem* items_host, int count, size_t total_tiles, int src_fmt,
+                                     int dst_fmt, cudaStream_t stream);
 // tiles one tensor of `nunits` lane units occupies in the batched kernel's tile space
 size_t ss_batched_tiles(size_t nunits);
 

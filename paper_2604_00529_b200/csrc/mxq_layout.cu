@@ -7,8 +7,9 @@
 // mxq_tile_scales re-orders stored scale bytes in a pass of its own; mxq_quantize_tiled and
 // mxq_slice_scale_tiled are Q_f and Slice-and-Scale with the scale bytes written in that order by the
 // producing kernel itself (put_scale in mxq_kernels.cuh), which saves the pass.
-#include "mxq_access.cuh"
-#include "mxq_codec.cuh"
+#include <vector>
+
+#include "mxq_kernels.cuh"
 #include "mxq_launch.h"
 
 namespace mxq {
@@ -136,6 +137,58 @@ int mxq_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t rows,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (int rc = clear_partial_tiles(out_tiled_scales, rows, kblocks, s)) return rc;
     return launch_slice_scale_tiled(codes, scales, n, src_fmt, dst_fmt, out_codes, out_tiled_scales, kblocks, s);
+}
+
+int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item* items, int count, int block, int src_fmt, int dst_fmt,
+                                  mxq_stream stream)
+{
+    if (fmt_info(src_fmt).kind != KIND_FP || fmt_info(dst_fmt).kind != KIND_FP) return MXQ_ERR_FORMAT;
+    if (block != 32) return MXQ_ERR_BLOCK;
+    if (!ss_pair_ok(src_fmt, dst_fmt)) return MXQ_ERR_PAIR;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+    // every item is checked before anything is enqueued
+    for (int i = 0; i < count; ++i) {
+        const mxq_ss_tiled_item& it = items[i];
+        size_t n;
+        uint32_t kblocks = 0;
+        if (int rc = check_tiled(it.rows, it.cols, block, &n, &kblocks)) return rc;
+        if (n == 0) continue;
+        if (!it.codes || !it.scales || !it.out_codes || !it.out_tiled_scales) return MXQ_ERR_NULL;
+        if (!aligned(it.codes, 32) || !aligned(it.out_codes, 32) || !aligned(it.scales, 16) ||
+            !aligned(it.out_tiled_scales, 16))
+            return MXQ_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<SsTiledDeviceItem> chunk;
+    chunk.reserve(kSsTiledItemsMax);
+    size_t tiles = 0;
+    auto flush = [&]() -> int {
+        if (chunk.empty()) return MXQ_OK;
+        const int rc = launch_slice_scale_tiled_batched(chunk.data(), (int)chunk.size(), tiles, src_fmt, dst_fmt, s);
+        chunk.clear();
+        tiles = 0;
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const mxq_ss_tiled_item& it = items[i];
+        if (it.rows == 0 || it.cols == 0) continue;
+        const uint32_t kblocks = (uint32_t)(it.cols / 32);
+        if (int rc = clear_partial_tiles(it.out_tiled_scales, it.rows, kblocks, s)) return rc;
+        SsTiledDeviceItem d;
+        d.codes = static_cast<const uint8_t*>(it.codes);
+        d.scales = it.scales;
+        d.out_codes = static_cast<uint8_t*>(it.out_codes);
+        d.out_scales = make_tiled_scales(it.out_tiled_scales, kblocks);
+        d.nunits = it.rows * it.cols / 32;
+        d.tile_begin = tiles;
+        tiles += ss_batched_tiles(d.nunits);
+        chunk.push_back(d);
+        if ((int)chunk.size() == kSsTiledItemsMax)
+            if (int rc = flush()) return rc;
+    }
+    return flush();
 }
 
 }  // extern "C"

@@ -71,6 +71,20 @@ int run_params(const SsDeviceItem* items_host, int count, size_t total_tiles, cu
     }
 }
 
+template <class FH, class FL>
+int run_tiled_params(const SsTiledDeviceItem* items_host, int count, size_t total_tiles, cudaStream_t stream)
+{
+    if constexpr (ss_pair_ok(FH::id, FL::id) && FL::kind == KIND_FP) {
+        SsTiledItemBlock<kSsTiledItemsMax> blk;
+        for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
+        for (int i = count; i < kSsTiledItemsMax; ++i) blk.items[i] = SsTiledDeviceItem{};
+        auto kern = slice_scale_tiled_batched_kernel<FH, FL, kU, kThreads, kSsTiledItemsMax>;
+        return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
+    } else {
+        return MXQ_ERR_PAIR;
+    }
+}
+
 }  // namespace
 
 size_t ss_batched_tiles(size_t nunits) { return (nunits + 32 * kU - 1) / (32 * kU); }
@@ -90,6 +104,16 @@ int launch_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t n,
     const TiledScales sink = make_tiled_scales(out_tiled, kblocks);
     MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
         MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_single_tiled<FH, FL>(codes, scales, n, out_codes, sink, stream); });
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+int launch_slice_scale_tiled_batched(const SsTiledDeviceItem* items_host, int count, size_t total_tiles, int src_fmt,
+                                     int dst_fmt, cudaStream_t stream)
+{
+    if (count > kSsTiledItemsMax) return MXQ_ERR_SIZE;
+    MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_tiled_params<FH, FL>(items_host, count, total_tiles, stream); });
     });
     return MXQ_ERR_FORMAT;
 }

@@ -98,6 +98,22 @@ def test_argument_checks_answer_on_the_host(L):
     assert st(A, A, 2, 80, 32, F["e4m3"], F["e2m1"], A, A, None) == E_SIZE
     assert st(A, None, 2, 64, 32, F["e4m3"], F["e2m1"], A, A, None) == E_NULL
     assert st(A, A, 2, 64, 32, F["e4m3"], F["e2m1"], A + 16, A, None) == E_ALIGN
+    stb = L.mxq_slice_scale_tiled_batched           # (items, count, block, src, dst, stream)
+    assert stb(None, 0, 32, F["e4m3"], F["e2m1"], None) == OK
+    assert stb(None, 2, 32, F["e4m3"], F["e2m1"], None) == E_NULL
+    assert stb(None, -1, 32, F["e4m3"], F["e2m1"], None) == E_SIZE
+    assert stb(None, 2, 64, F["e4m3"], F["e2m1"], None) == E_BLOCK
+    assert stb(None, 2, 32, F["int8"], F["int4"], None) == E_FORMAT
+    assert stb(None, 2, 32, F["e2m1"], F["e4m3"], None) == E_PAIR
+    from paper_2604_00529_b200.binding import _TiledItem
+    one = (_TiledItem * 1)(_TiledItem(A, A, 2, 48, A, A))
+    assert stb(one, 1, 32, F["e4m3"], F["e2m1"], None) == E_SIZE
+    one = (_TiledItem * 1)(_TiledItem(A, A, 2, 64, A, None))
+    assert stb(one, 1, 32, F["e4m3"], F["e2m1"], None) == E_NULL
+    one = (_TiledItem * 1)(_TiledItem(A, A, 2, 64, A, A + 8))
+    assert stb(one, 1, 32, F["e4m3"], F["e2m1"], None) == E_ALIGN
+    one = (_TiledItem * 1)(_TiledItem(None, None, 0, 64, None, None))
+    assert stb(one, 1, 32, F["e4m3"], F["e2m1"], None) == OK                 # an empty matrix: nothing to do
     dq = L.mxq_dequantize
     assert dq(A, A, 64, F["int4"], 32, A, 5, None) == E_FORMAT
     assert dq(A, None, 64, F["int4"], 32, A, 0, None) == E_NULL

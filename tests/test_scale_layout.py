@@ -114,6 +114,40 @@ def test_gpu_slice_scale_tiled_equals_slice_scale_then_tile(rows, kb):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("count", [1, 5, 256, 257, 600])
+def test_gpu_slice_scale_tiled_batched_matches_oracle(count):
+    """Many small matrices of assorted shapes in one call (more than one launch beyond 256 items), with an
+    empty one among them; every output against the oracle's Slice-and-Scale followed by its tiling."""
+    rng = np.random.default_rng(count)
+    shapes = [(int(rng.integers(1, 200)), 32 * int(rng.integers(1, 12))) for _ in range(count)]
+    if count > 3:
+        shapes[2] = (0, 64)
+    items, want = [], []
+    for k, (rows, cols) in enumerate(shapes):
+        kb = cols // 32
+        n = rows * cols
+        bits = _bf16_matrix(rows, cols, 1000 * count + k) if n else np.zeros(0, np.uint16)
+        ac, as_ = orc.quantize(bits, "e4m3", 32) if n else (np.zeros(0, np.uint8), np.zeros(0, np.uint8))
+        wc, ws = orc.slice_scale(ac, as_, "e4m3", "e2m1", 32) if n else (ac, as_)
+        nbytes = mxq.tiled_scales_bytes(rows, kb) if n else 0
+        # tensors are padded so that every device pointer keeps the 32-byte alignment inside one arena
+        items.append((torch.from_numpy(orc.pack(ac, 8)).cuda() if n else torch.empty(32, dtype=torch.uint8, device="cuda"),
+                      torch.from_numpy(as_).cuda() if n else torch.empty(32, dtype=torch.uint8, device="cuda"),
+                      rows, cols,
+                      torch.full((max(n // 2, 32),), 0xA5, dtype=torch.uint8, device="cuda"),
+                      torch.full((max(nbytes, 32),), 0xA5, dtype=torch.uint8, device="cuda")))
+        want.append((orc.pack(wc, 4), orc.tile_scales(ws.reshape(rows, kb), rows, kb) if n else None, n, nbytes))
+    mxq.slice_scale_tiled_batched(items, "e4m3", "e2m1", 32)
+    torch.cuda.synchronize()
+    for k, ((_, _, rows, cols, oc, ot), (wc, wt, n, nbytes)) in enumerate(zip(items, want)):
+        if n == 0:
+            assert bool((oc == 0xA5).all()) and bool((ot == 0xA5).all()), k
+            continue
+        assert np.array_equal(oc.cpu().numpy()[:n // 2], wc), (k, rows, cols)
+        assert np.array_equal(ot.cpu().numpy()[:nbytes], wt), (k, rows, cols)
+
+
+@pytest.mark.gpu
 def test_gpu_tiled_entry_points_full_size_workload():
     """BF16 8192 x 8192 (the bench's workload): fused outputs equal the two-pass outputs byte for byte
     (the two-pass path is compared with the oracle at this size elsewhere)."""
