@@ -396,7 +396,8 @@ def run_cuda(args):
     top_gbs = OP_BYTES[top_name] * n / (iso_ms[top] * 1e-3) / 1e9
     traffic = NCU_TRAFFIC.get(top_name) if kernel_sources_digest() == NCU_TRAFFIC_SOURCES else None
 
-    cpu = cpu_baseline(x_bits)
+    # the oracle is timed beside the one-GPU run only: at N > 1 every rank's GPU would be held meanwhile
+    cpu = cpu_baseline(x_bits) if world == 1 else None
     line = {
         "metric": "mx_requant_hot_path_hbm_gbs", "value": round(value, 1), "unit": "GB/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5),
