@@ -309,6 +309,7 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
         stage = stage_area + (threadIdx.x >> 5) * (32 * U * OB);
     }
 
+    prefetch_tile<U, 32>(src, warp, nunits);
     pdl_acquire();
     if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
@@ -505,6 +506,7 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    prefetch_tile<U, 32>(src, tile, nunits);
     pdl_acquire();
     if (tile * (32 * U) < nunits) fake_quant_tile<T, F, BLOCK, MODE, U>(src, nunits, dst, tile);
 }
@@ -529,15 +531,17 @@ fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count,
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    pdl_acquire();
-    if (tile >= total_tiles) return;                      // whole warps leave together
-    int lo = 0, hi = count - 1;
+    // the item table is a kernel parameter, so the search may run before the dependency wait
+    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         if (blk.items[mid].tile_begin <= tile) lo = mid;
         else hi = mid - 1;
     }
     const FqDeviceItem& t = blk.items[lo];
+    if (tile < total_tiles) prefetch_tile<U, 32>(t.src, tile - t.tile_begin, t.nunits);
+    pdl_acquire();
+    if (tile >= total_tiles) return;                      // whole warps leave together
     fake_quant_tile<T, F, BLOCK, MODE, U>(t.src, t.nunits, t.dst, tile - t.tile_begin);
 }
 
@@ -819,6 +823,7 @@ slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
+    prefetch_tile<U, 4 * FH::bits>(codes, tile, nunits);
     pdl_acquire();
     if (tile * (32 * U) < nunits)
         slice_scale_tile<FH, FL, U>(codes, scales, nunits, nscales, out_codes, out_scales, tile, stage);
@@ -848,6 +853,7 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
         __shared__ __align__(16) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
         stage2 = area2 + (threadIdx.x >> 5) * (32 * U * OB2);
     }
+    prefetch_tile<U, IB>(codes, tile, nunits);
     pdl_acquire();
     if (tile * (32 * U) >= nunits) return;                     // whole warps leave together
     uint32_t w[U][NWI];
@@ -959,15 +965,16 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
-    pdl_acquire();
-    if (tile >= total_tiles) return;
-    int lo = 0, hi = count - 1;
+    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;       // parameters: readable before the wait
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         if (blk.items[mid].tile_begin <= tile) lo = mid;
         else hi = mid - 1;
     }
     const SsDeviceItem& t = blk.items[lo];
+    if (tile < total_tiles) prefetch_tile<U, 4 * FH::bits>(t.codes, tile - t.tile_begin, t.nunits);
+    pdl_acquire();
+    if (tile >= total_tiles) return;
     slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin,
                                 stage);
 }
@@ -996,15 +1003,16 @@ slice_scale_tiled_batched_kernel(const __grid_constant__ SsTiledItemBlock<K> blk
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
-    pdl_acquire();
-    if (tile >= total_tiles) return;
-    int lo = 0, hi = count - 1;
+    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;       // parameters: readable before the wait
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
         if (blk.items[mid].tile_begin <= tile) lo = mid;
         else hi = mid - 1;
     }
     const SsTiledDeviceItem& t = blk.items[lo];
+    if (tile < total_tiles) prefetch_tile<U, 4 * FH::bits>(t.codes, tile - t.tile_begin, t.nunits);
+    pdl_acquire();
+    if (tile >= total_tiles) return;
     slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nunits, t.out_codes, t.out_scales, tile - t.tile_begin,
                                 stage);
 }
@@ -1173,6 +1181,7 @@ copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict_
     const int lane = threadIdx.x & 31;
     const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    prefetch_tile<U, 32>(src, warp, nunits);
     pdl_acquire();
     if (const size_t tile = warp; tile < ntiles) {
         const size_t u0 = tile * (32 * U) + lane;
