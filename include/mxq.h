@@ -21,8 +21,10 @@
  *   - Work goes to the CURRENT device, which must be the one the pointers belong to.  Kernels
  *     are launched with programmatic stream serialization allowed, so that a kernel's blocks
  *     can become resident while the previous kernel of the stream drains; each kernel waits
- *     for that previous kernel to complete before its first global memory access, so the
- *     ordering a stream guarantees is unchanged for every buffer.
+ *     for that previous kernel to complete before its first load or store, so the ordering a
+ *     stream guarantees is unchanged for every buffer.  (Before that wait a kernel may issue
+ *     L2 prefetches for its input buffers, which return no data; the input pointers must
+ *     therefore be valid device addresses when the call is made, as they must be anyway.)
  *   - `n` is the number of elements; it must be a multiple of `block`.  Blocks are runs
  *     of `block` consecutive elements of the flat array (for a row-major matrix whose inner
  *     dimension is a multiple of `block`: along the row).  n == 0 returns MXQ_OK at once.
