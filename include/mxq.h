@@ -223,11 +223,9 @@ int mxq_fake_quant_bwd(const void *grad_out, int dtype, size_t n, void *grad_in,
  * Whole-model on-the-fly conversion (Sec. 3.5, Inference): mxq_slice_scale over `count`
  * tensors in one launch.  `items` is a HOST array; every pointer inside is a device
  * pointer with the same requirements as in mxq_slice_scale; the host array may be freed
- * as soon as the call returns.  Up to 512 non-empty tensors travel in the kernel's own
- * parameter space (no allocation, no copy).  Beyond that the item table is copied to a
- * device-side table owned by the library (grown with cudaMalloc on first use or when
- * `count` exceeds its capacity, reused afterwards); such calls are ordered by `stream`
- * and must not run concurrently on different streams.
+ * as soon as the call returns.  The item table travels in the kernel's own parameter
+ * space, 512 non-empty tensors per launch (more tensors: more launches); nothing is
+ * allocated or copied and no state is shared between calls.
  */
 typedef struct {
     const void *codes;
@@ -267,7 +265,9 @@ int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item *items, int count, int
  * never stall, and cudaMalloc / cudaFree wait for the device.  For them the item table lives in a
  * fixed array inside the library image: MXQ_STATIC_BATCH_MAX items, 56 KiB, present on every GPU
  * that loads libmxq until the process exits.  This call makes no cudaMalloc, cudaFree or other
- * allocating call, on the device or on the host heap.
+ * allocating call, on the device or on the host heap, and converts up to MXQ_STATIC_BATCH_MAX
+ * tensors in one launch.  (mxq_slice_scale_batched allocates nothing on the device either, but it
+ * builds its launch tables on the host heap and needs one launch per 512 tensors.)
  *   - Arguments, checks and results are those of mxq_slice_scale_batched (block must be 32, 64 or
  *     128); in addition count > MXQ_STATIC_BATCH_MAX returns MXQ_ERR_SIZE and launches nothing.
  *   - The first call on each device looks up the array's device address (with that device current)

@@ -1,6 +1,5 @@
 // The C ABI of libmxq (declared in include/mxq.h): argument validation on the host, then the
 // per-operation launchers.  Nothing here synchronises the device.
-#include <mutex>
 #include <vector>
 
 #include "mxq_kernels.cuh"
@@ -9,17 +8,6 @@
 namespace mxq {
 
 namespace {
-
-constexpr int kMaxDevices = 64;
-
-std::mutex g_mutex;
-
-int current_device()
-{
-    int d = 0;
-    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) return -1;
-    return d;
-}
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -34,13 +22,6 @@ int check_sizes(size_t n, int block)
     if (n % (size_t)block) return MXQ_ERR_SIZE;
     return MXQ_OK;
 }
-
-// Device-side item table of the batched conversion: library-owned scratch, one per device.
-struct ItemTable {
-    SsDeviceItem* dev = nullptr;
-    int capacity = 0;
-};
-ItemTable g_table[kMaxDevices];
 
 }  // namespace
 
@@ -250,37 +231,19 @@ int mxq_slice_scale_batched(const mxq_ss_item* items, int count, int block, int 
     }
     if (host.empty()) return MXQ_OK;
 
+    // the item table rides in the kernel's parameter space, kSsParamItemsMax tensors per launch: nothing
+    // to allocate or copy, no state shared between calls; larger sets take several launches (each
+    // launch's tiles are numbered from zero)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // up to kSsParamItemsMax tensors travel in the kernel's parameter space: nothing to allocate or copy
-    if ((int)host.size() <= kSsParamItemsMax)
-        return launch_slice_scale_batched_params(host.data(), (int)host.size(), tiles, src_fmt, dst_fmt, s);
-    const int dev = current_device();
-    if (dev < 0) return MXQ_ERR_CUDA;
-    SsDeviceItem* table = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        ItemTable& t = g_table[dev];
-        if (t.capacity < (int)host.size()) {
-            // grow: the old table may still be read by an earlier launch on this stream, so free it
-            // only after that work has drained
-            if (t.dev) {
-                if (cudaStreamSynchronize(s) != cudaSuccess) return MXQ_ERR_CUDA;
-                cudaFree(t.dev);
-                t.dev = nullptr;
-                t.capacity = 0;
-            }
-            int cap = 256;
-            while (cap < (int)host.size()) cap *= 2;
-            if (cudaMalloc(&t.dev, sizeof(SsDeviceItem) * (size_t)cap) != cudaSuccess) return MXQ_ERR_CUDA;
-            t.capacity = cap;
-        }
-        table = t.dev;
+    for (size_t first = 0; first < host.size(); first += kSsParamItemsMax) {
+        const size_t cnt = host.size() - first < (size_t)kSsParamItemsMax ? host.size() - first : (size_t)kSsParamItemsMax;
+        const size_t base = host[first].tile_begin;
+        for (size_t i = first; i < first + cnt; ++i) host[i].tile_begin -= base;
+        const size_t end = first + cnt < host.size() ? host[first + cnt].tile_begin : tiles;
+        if (int rc = launch_slice_scale_batched_params(host.data() + first, (int)cnt, end - base, src_fmt, dst_fmt, s))
+            return rc;
     }
-    // pageable source: the runtime stages the bytes before returning, so `host` may go out of scope
-    if (cudaMemcpyAsync(table, host.data(), sizeof(SsDeviceItem) * host.size(), cudaMemcpyHostToDevice, s) !=
-        cudaSuccess)
-        return MXQ_ERR_CUDA;
-    return launch_slice_scale_batched(table, (int)host.size(), tiles, src_fmt, dst_fmt, s);
+    return MXQ_OK;
 }
 
 }  // extern "C"

@@ -186,7 +186,7 @@ def test_slice_scale_batched_matches_oracle():
 @pytest.mark.parametrize("count", [64, 65, 512, 513, 700])
 def test_slice_scale_batched_item_counts(count):
     """Item counts on both sides of the limits where the item table changes its way to the kernel
-    (small and large kernel-parameter blocks, device-side table)."""
+    (small and large kernel-parameter blocks, more than one launch)."""
     rng = np.random.default_rng(count)
     sizes = (64 * rng.integers(1, 8, count)).tolist()          # 64-element multiples keep every pointer 32-byte aligned
     total = int(sum(sizes))
@@ -437,7 +437,7 @@ def test_tensor_level_mse_study_on_gpu():
 
 def test_two_streams_run_independent_conversions():
     """The same calls issued on two non-default streams at once give what they give alone (every
-    entry point takes its stream from the caller; only the >512-tensor batched path shares state)."""
+    entry point takes its stream from the caller; only the fixed-table batched entry point shares state)."""
     x1 = inputs.to_bf16_bits(_mixed_f32(4099, 21))
     x2 = inputs.to_bf16_bits(_mixed_f32(4099, 22))
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
