@@ -17,6 +17,7 @@ int run(const FqDeviceItem* items_host, int count, size_t total_tiles, cudaStrea
         FqItemBlock<kFqBatchItemsMax> blk;
         for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
         for (int i = count; i < kFqBatchItemsMax; ++i) blk.items[i] = FqDeviceItem{};
+        build_tile_index(blk.index, items_host, count, total_tiles);
         auto kern = fake_quant_batched_kernel<T, F, BLOCK, MODE, kU, kThreads, kFqBatchItemsMax>;
         return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
     }

@@ -511,6 +511,48 @@ fake_quant_kernel(const uint8_t* src, size_t nunits, uint8_t* dst)   // dst may 
     if (tile * (32 * U) < nunits) fake_quant_tile<T, F, BLOCK, MODE, U>(src, nunits, dst, tile);
 }
 
+// Which tensor of a batch owns a tile.  The batched kernels lay the tiles of all tensors end to end;
+// the items (sorted by tile_begin) ride in the kernel parameters.  A plain binary search over a few
+// hundred items costs eight dependent constant-memory reads and some fifty instructions per warp
+// tile, 10 - 20 % of such a kernel.  The host therefore adds a coarse index: the tile space is cut
+// into at most 256 segments of 2^shift tiles, coarse[k] is the item that owns the first tile of
+// segment k (coarse[last + 1] the last item), and a tile's owner lies between the entries of its
+// segment's two ends -- usually the same item or neighbours, so the search that remains takes zero
+// to two steps.
+struct TileIndex {
+    uint32_t shift;
+    uint16_t coarse[258];
+};
+
+template <class ITEM>
+inline void build_tile_index(TileIndex& ix, const ITEM* items, int count, size_t total_tiles)
+{
+    ix.shift = 0;
+    while ((total_tiles >> ix.shift) > 255) ++ix.shift;
+    const size_t nseg = total_tiles ? ((total_tiles - 1) >> ix.shift) + 1 : 1;
+    int it = 0;
+    for (size_t k = 0; k < nseg; ++k) {
+        const size_t first = k << ix.shift;
+        while (it + 1 < count && items[it + 1].tile_begin <= first) ++it;
+        ix.coarse[k] = (uint16_t)it;
+    }
+    for (size_t k = nseg; k < 258; ++k) ix.coarse[k] = (uint16_t)(count - 1);
+}
+
+// `items` is an array inside a __grid_constant__ kernel parameter; tile < total_tiles.
+template <class ITEM>
+__device__ __forceinline__ int find_item(const ITEM* items, const TileIndex& ix, size_t tile)
+{
+    const uint32_t k = (uint32_t)(tile >> ix.shift);
+    int lo = ix.coarse[k], hi = ix.coarse[k + 1];
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (items[mid].tile_begin <= tile) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+
 // The fake-quant of a whole set of tensors (every quantized weight of a model in one QAT step, Eq. 6)
 // in one launch: the tiles of all tensors laid end to end, the item table in the kernel's parameters.
 struct FqDeviceItem {
@@ -523,6 +565,7 @@ struct FqDeviceItem {
 template <int K>
 struct FqItemBlock {
     FqDeviceItem items[K];
+    TileIndex index;
 };
 
 template <class T, class F, int BLOCK, int MODE, int U, int THREADS, int K>
@@ -531,14 +574,8 @@ fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count,
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    // the item table is a kernel parameter, so the search may run before the dependency wait
-    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (blk.items[mid].tile_begin <= tile) lo = mid;
-        else hi = mid - 1;
-    }
-    const FqDeviceItem& t = blk.items[lo];
+    // the item table is a kernel parameter, so the lookup may run before the dependency wait
+    const FqDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
     if (tile < total_tiles) prefetch_tile<U, 32>(t.src, tile - t.tile_begin, t.nunits);
     pdl_acquire();
     if (tile >= total_tiles) return;                      // whole warps leave together
@@ -951,11 +988,12 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
 }
 
 // The same launch with the item table carried in the kernel's parameter space (K items, 56 bytes
-// each: K = 64 stays under the classic 4 KB of parameters, K = 512 uses the 32 KB that sm_70 and
-// later allow).  No device buffer, no host-to-device copy in front of the kernel.
+// each, plus the coarse index: K = 64 stays near the classic 4 KB of parameters, K = 512 uses the
+// 32 KB that sm_70 and later allow).  No device buffer, no host-to-device copy in front of the kernel.
 template <int K>
 struct SsItemBlock {
     SsDeviceItem items[K];
+    TileIndex index;
 };
 
 template <class FH, class FL, int U, int THREADS, int K>
@@ -965,13 +1003,8 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
-    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;       // parameters: readable before the wait
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (blk.items[mid].tile_begin <= tile) lo = mid;
-        else hi = mid - 1;
-    }
-    const SsDeviceItem& t = blk.items[lo];
+    // parameters: readable before the wait
+    const SsDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
     if (tile < total_tiles) prefetch_tile<U, 4 * FH::bits>(t.codes, tile - t.tile_begin, t.nunits);
     pdl_acquire();
     if (tile >= total_tiles) return;
@@ -994,6 +1027,7 @@ struct SsTiledDeviceItem {
 template <int K>
 struct SsTiledItemBlock {
     SsTiledDeviceItem items[K];
+    TileIndex index;
 };
 
 template <class FH, class FL, int U, int THREADS, int K>
@@ -1003,13 +1037,8 @@ slice_scale_tiled_batched_kernel(const __grid_constant__ SsTiledItemBlock<K> blk
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     uint8_t* stage = slice_scale_stage<FL, U, THREADS>();
-    int lo = 0, hi = tile < total_tiles ? count - 1 : 0;       // parameters: readable before the wait
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (blk.items[mid].tile_begin <= tile) lo = mid;
-        else hi = mid - 1;
-    }
-    const SsTiledDeviceItem& t = blk.items[lo];
+    // parameters: readable before the wait
+    const SsTiledDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
     if (tile < total_tiles) prefetch_tile<U, 4 * FH::bits>(t.codes, tile - t.tile_begin, t.nunits);
     pdl_acquire();
     if (tile >= total_tiles) return;

@@ -61,6 +61,7 @@ int run_params(const SsDeviceItem* items_host, int count, size_t total_tiles, cu
             SsItemBlock<K> blk;
             for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
             for (int i = count; i < K; ++i) blk.items[i] = SsDeviceItem{};
+            build_tile_index(blk.index, items_host, count, total_tiles);
             auto kern = slice_scale_batched_param_kernel<FH, FL, kU, kThreads, K>;
             return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
         };
@@ -78,6 +79,7 @@ int run_tiled_params(const SsTiledDeviceItem* items_host, int count, size_t tota
         SsTiledItemBlock<kSsTiledItemsMax> blk;
         for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
         for (int i = count; i < kSsTiledItemsMax; ++i) blk.items[i] = SsTiledDeviceItem{};
+        build_tile_index(blk.index, items_host, count, total_tiles);
         auto kern = slice_scale_tiled_batched_kernel<FH, FL, kU, kThreads, kSsTiledItemsMax>;
         return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
     } else {
