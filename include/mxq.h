@@ -263,8 +263,8 @@ int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item *items, int count, int
  * processes give all of HBM to a pool of their own at start-up, so a cudaMalloc made behind their
  * back fails or takes memory that was promised elsewhere; others run a loop where the host must
  * never stall, and cudaMalloc / cudaFree wait for the device.  For them the item table lives in a
- * fixed array inside the library image: MXQ_STATIC_BATCH_MAX items, 56 KiB, present on every GPU
- * that loads libmxq until the process exits.  This call makes no cudaMalloc, cudaFree or other
+ * fixed array inside the library image: MXQ_STATIC_BATCH_MAX items and a small index, 57 KiB,
+ * present on every GPU that loads libmxq until the process exits.  This call makes no cudaMalloc, cudaFree or other
  * allocating call, on the device or on the host heap, and converts up to MXQ_STATIC_BATCH_MAX
  * tensors in one launch.  (mxq_slice_scale_batched allocates nothing on the device either, but it
  * builds its launch tables on the host heap and needs one launch per 512 tensors.)

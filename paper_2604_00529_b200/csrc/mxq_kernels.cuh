@@ -968,7 +968,8 @@ struct SsDeviceItem {
 // SMs idle.
 template <class FH, class FL, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
-slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, size_t total_tiles)
+slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, const TileIndex* __restrict__ index, int count,
+                           size_t total_tiles)
 {
     pdl_release();
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
@@ -976,13 +977,8 @@ slice_scale_batched_kernel(const SsDeviceItem* __restrict__ items, int count, si
     pdl_acquire();
     if (tile >= total_tiles) return;
     // items are sorted by tile_begin: the last one that starts at or before this tile owns it
-    int lo = 0, hi = count - 1;
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (items[mid].tile_begin <= tile) lo = mid;
-        else hi = mid - 1;
-    }
-    const SsDeviceItem t = items[lo];
+    // (table and index are device memory written by the copy in front of this launch: read after the wait)
+    const SsDeviceItem t = items[find_item(items, *index, tile)];
     slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin,
                                 stage);
 }

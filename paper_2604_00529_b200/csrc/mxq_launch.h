@@ -49,8 +49,9 @@ int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
 
 // Batched Slice-and-Scale over a device-resident item table (see mxq_kernels.cuh: SsDeviceItem).
 struct SsDeviceItem;
-int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t total_tiles, int src_fmt,
-                               int dst_fmt, cudaStream_t stream);
+struct TileIndex;
+int launch_slice_scale_batched(const SsDeviceItem* items_dev, const TileIndex* index_dev, int count, size_t total_tiles,
+                               int src_fmt, int dst_fmt, cudaStream_t stream);
 // The same launch with the items (a HOST array here) passed in the kernel's parameter space; count
 // must not exceed kSsParamItemsMax.
 constexpr int kSsParamItemsMax = 512;

@@ -42,11 +42,13 @@ int run_single_tiled(const void* codes, const uint8_t* scales, size_t n, void* o
 }
 
 template <class FH, class FL>
-int run_table(const SsDeviceItem* items_dev, int count, size_t total_tiles, cudaStream_t stream)
+int run_table(const SsDeviceItem* items_dev, const TileIndex* index_dev, int count, size_t total_tiles,
+              cudaStream_t stream)
 {
     if constexpr (ss_pair_ok(FH::id, FL::id)) {
         auto kern = slice_scale_batched_kernel<FH, FL, kU, kThreads>;
-        return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, items_dev, count, total_tiles);
+        return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, items_dev, index_dev, count,
+                             total_tiles);
     } else {
         return MXQ_ERR_PAIR;
     }
@@ -120,11 +122,11 @@ int launch_slice_scale_tiled_batched(const SsTiledDeviceItem* items_host, int co
     return MXQ_ERR_FORMAT;
 }
 
-int launch_slice_scale_batched(const SsDeviceItem* items_dev, int count, size_t total_tiles, int src_fmt,
-                               int dst_fmt, cudaStream_t stream)
+int launch_slice_scale_batched(const SsDeviceItem* items_dev, const TileIndex* index_dev, int count, size_t total_tiles,
+                               int src_fmt, int dst_fmt, cudaStream_t stream)
 {
     MXQ_DISPATCH_FORMAT_AS(src_fmt, FH, {
-        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_table<FH, FL>(items_dev, count, total_tiles, stream); });
+        MXQ_DISPATCH_FORMAT_AS(dst_fmt, FL, { return run_table<FH, FL>(items_dev, index_dev, count, total_tiles, stream); });
     });
     return MXQ_ERR_FORMAT;
 }

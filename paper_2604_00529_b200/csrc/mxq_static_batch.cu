@@ -5,6 +5,7 @@
 // Who needs this: a serving process that has handed the whole HBM to its own pool (weights, KV
 // cache) so that a stray cudaMalloc fails or eats into a budget somebody else planned; and a
 // latency-critical loop, where cudaMalloc / cudaFree stall the host until the device is idle.
+#include <cstddef>
 #include <mutex>
 
 #include "mxq_kernels.cuh"
@@ -15,17 +16,23 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 
-// The table itself: MXQ_STATIC_BATCH_MAX items of 56 bytes = 56 KiB on every GPU that loads the
-// library, for the life of the process.  In host code this name is only a handle for
+// What one call hands to the kernel: the coarse index over the tile space, then the items.
+struct StaticTable {
+    TileIndex index;
+    SsDeviceItem items[MXQ_STATIC_BATCH_MAX];
+};
+
+// The table itself: MXQ_STATIC_BATCH_MAX items of 56 bytes and the 520-byte index = 57 KiB on every GPU
+// that loads the library, for the life of the process.  In host code this name is only a handle for
 // cudaGetSymbolAddress; it is not a device address and must never be handed to a kernel.
-static __device__ __align__(256) unsigned char g_static_items[MXQ_STATIC_BATCH_MAX * sizeof(SsDeviceItem)];
+static __device__ __align__(256) unsigned char g_static_items[sizeof(StaticTable)];
 
 std::mutex g_static_mutex;
-SsDeviceItem* g_static_table[kMaxDevices];      // device address of g_static_items, per device
+StaticTable* g_static_table[kMaxDevices];       // device address of g_static_items, per device
 
 // Device address of the table on the current device; looked up once per device, with that device
 // current (the caller's), on the first call that reaches here.
-int static_table(SsDeviceItem** out)
+int static_table(StaticTable** out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MXQ_ERR_CUDA;
@@ -36,7 +43,7 @@ int static_table(SsDeviceItem** out)
             (void)cudaGetLastError();
             return MXQ_ERR_CUDA;
         }
-        g_static_table[dev] = static_cast<SsDeviceItem*>(p);
+        g_static_table[dev] = static_cast<StaticTable*>(p);
     }
     *out = g_static_table[dev];
     return MXQ_OK;
@@ -61,7 +68,8 @@ extern "C" int mxq_slice_scale_batched_static(const mxq_ss_item* items, int coun
     if (!items) return MXQ_ERR_NULL;
 
     // host copy of the table on the stack: no heap, no pinned allocation
-    SsDeviceItem host[MXQ_STATIC_BATCH_MAX];
+    StaticTable staged;
+    SsDeviceItem* host = staged.items;
     int used = 0;
     size_t tiles = 0;
     for (int i = 0; i < count; ++i) {
@@ -84,14 +92,15 @@ extern "C" int mxq_slice_scale_batched_static(const mxq_ss_item* items, int coun
     }
     if (used == 0) return MXQ_OK;
 
-    SsDeviceItem* table = nullptr;
+    build_tile_index(staged.index, host, used, tiles);
+    StaticTable* table = nullptr;
     if (int rc = static_table(&table)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // Entries [0, used) are rewritten by every call and the kernel reads no others, so nothing in
     // the table has to start from zero.  The source is pageable stack memory: the runtime has
     // staged the bytes by the time this returns.
-    if (cudaMemcpyAsync(table, host, sizeof(SsDeviceItem) * (size_t)used, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return MXQ_ERR_CUDA;
-    return launch_slice_scale_batched(table, used, tiles, src_fmt, dst_fmt, s);
+    const size_t nbytes = offsetof(StaticTable, items) + sizeof(SsDeviceItem) * (size_t)used;
+    if (cudaMemcpyAsync(table, &staged, nbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MXQ_ERR_CUDA;
+    return launch_slice_scale_batched(table->items, &table->index, used, tiles, src_fmt, dst_fmt, s);
 }
 #pragma GCC visibility pop
