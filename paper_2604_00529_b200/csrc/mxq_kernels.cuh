@@ -66,14 +66,24 @@ inline TiledScales make_tiled_scales(uint8_t* base, uint32_t kblocks)      // 1 
     return TiledScales{base, kblocks, (uint32_t)m, s < 1 ? s : 1u, s > 1 ? s - 1 : 0u, (kblocks + 3) / 4};
 }
 
-__device__ __forceinline__ void put_scale(const TiledScales& t, size_t blk, uint32_t byte)
+// Byte offset of block `blk` (row-major index, below 2^32) inside the tiled buffer.
+__host__ __device__ __forceinline__ size_t tiled_scale_offset(const TiledScales& t, size_t blk)
 {
     const uint32_t n = (uint32_t)blk;
+#ifdef __CUDA_ARCH__
     const uint32_t hi = __umulhi(t.magic, n);
+#else
+    const uint32_t hi = (uint32_t)(((uint64_t)t.magic * n) >> 32);
+#endif
     const uint32_t r = (hi + ((n - hi) >> t.shift1)) >> t.shift2;
     const uint32_t c = n - r * t.kblocks;
     const size_t tile = (size_t)(r >> 7) * t.col_tiles + (c >> 2);
-    t.base[tile * 512 + (r & 31u) * 16u + ((r >> 5) & 3u) * 4u + (c & 3u)] = (uint8_t)byte;
+    return tile * 512 + (r & 31u) * 16u + ((r >> 5) & 3u) * 4u + (c & 3u);
+}
+
+__device__ __forceinline__ void put_scale(const TiledScales& t, size_t blk, uint32_t byte)
+{
+    t.base[tiled_scale_offset(t, blk)] = (uint8_t)byte;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -541,7 +551,7 @@ inline void build_tile_index(TileIndex& ix, const ITEM* items, int count, size_t
 
 // `items` is an array inside a __grid_constant__ kernel parameter; tile < total_tiles.
 template <class ITEM>
-__device__ __forceinline__ int find_item(const ITEM* items, const TileIndex& ix, size_t tile)
+__host__ __device__ __forceinline__ int find_item(const ITEM* items, const TileIndex& ix, size_t tile)
 {
     const uint32_t k = (uint32_t)(tile >> ix.shift);
     int lo = ix.coarse[k], hi = ix.coarse[k + 1];
