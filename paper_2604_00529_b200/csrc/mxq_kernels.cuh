@@ -10,6 +10,9 @@
 //   dequantize            : to 16-bit outputs a unit is 32 element codes (64 B out); to FP32 it is 32 B
 //                           of output (8 elements), see dequantize_wide_kernel.
 //
+// Every kernel lets its successor start launching at once, asks L2 for its own input lines, and only
+// then waits for its predecessor (see pdl_release / prefetch_tile / pdl_acquire in mxq_access.cuh).
+//
 // All of them are bound by HBM traffic, with the integer/logic pipe (64 lanes per clock per SM) as
 // the second bound; the arithmetic below is shaped to stay under it: packed 16-bit maxima, round-down
 // FP32 adds instead of float->int conversions, four 8-bit codes per register (SWAR), per-byte signs

@@ -47,7 +47,8 @@ int launch_fake_quant_batched(const FqDeviceItem* items_host, int count, size_t 
 size_t fq_batched_tiles(size_t nunits);
 int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
 
-// Batched Slice-and-Scale over a device-resident item table (see mxq_kernels.cuh: SsDeviceItem).
+// Batched Slice-and-Scale over a device-resident item table and its coarse tile index (see
+// mxq_kernels.cuh: SsDeviceItem, TileIndex); used by the fixed-table entry point.
 struct SsDeviceItem;
 struct TileIndex;
 int launch_slice_scale_batched(const SsDeviceItem* items_dev, const TileIndex* index_dev, int count, size_t total_tiles,

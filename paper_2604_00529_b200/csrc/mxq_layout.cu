@@ -52,35 +52,9 @@ tile_scales_kernel(const uint8_t* __restrict__ scales, size_t rows, size_t kbloc
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-}  // namespace
-}  // namespace mxq
+inline size_t tiled_bytes(size_t rows, size_t kblocks) { return ((rows + 127) / 128) * ((kblocks + 3) / 4) * 512; }
 
-using namespace mxq;
-
-#pragma GCC visibility push(default)
-extern "C" {
-
-size_t mxq_tiled_scales_bytes(size_t rows, size_t kblocks)
-{
-    return ((rows + 127) / 128) * ((kblocks + 3) / 4) * 512;
-}
-
-int mxq_tile_scales(const uint8_t* scales, size_t rows, size_t kblocks, uint8_t* tiled, mxq_stream stream)
-{
-    if (rows == 0 || kblocks == 0) return MXQ_OK;
-    if (!scales || !tiled) return MXQ_ERR_NULL;
-    if (!aligned(scales, 16) || !aligned(tiled, 16)) return MXQ_ERR_ALIGN;
-    const size_t col_tiles = (kblocks + 3) / 4, ntiles = ((rows + 127) / 128) * col_tiles;
-    const int grid = grid_for_tiles(ntiles, kThreads);
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (kblocks % 4 == 0)
-        return launch_kernel(tile_scales_kernel<true>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
-    return launch_kernel(tile_scales_kernel<false>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
-}
-
-namespace {
-
-// Checks shared by the two fused entry points.  On MXQ_OK with *n == 0 there is nothing to do.
+// Checks shared by the fused entry points.  On MXQ_OK with *n == 0 there is nothing to do.
 int check_tiled(size_t rows, size_t cols, int block, size_t* n, uint32_t* kblocks)
 {
     *n = 0;
@@ -98,7 +72,7 @@ int check_tiled(size_t rows, size_t cols, int block, size_t* n, uint32_t* kblock
 int clear_partial_tiles(uint8_t* tiled, size_t rows, size_t kblocks, cudaStream_t s)
 {
     if (rows % 128 == 0 && kblocks % 4 == 0) return MXQ_OK;
-    if (cudaMemsetAsync(tiled, 0, mxq_tiled_scales_bytes(rows, kblocks), s) != cudaSuccess) {
+    if (cudaMemsetAsync(tiled, 0, tiled_bytes(rows, kblocks), s) != cudaSuccess) {
         (void)cudaGetLastError();
         return MXQ_ERR_CUDA;
     }
@@ -106,6 +80,28 @@ int clear_partial_tiles(uint8_t* tiled, size_t rows, size_t kblocks, cudaStream_
 }
 
 }  // namespace
+
+}  // namespace mxq
+
+using namespace mxq;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+size_t mxq_tiled_scales_bytes(size_t rows, size_t kblocks) { return tiled_bytes(rows, kblocks); }
+
+int mxq_tile_scales(const uint8_t* scales, size_t rows, size_t kblocks, uint8_t* tiled, mxq_stream stream)
+{
+    if (rows == 0 || kblocks == 0) return MXQ_OK;
+    if (!scales || !tiled) return MXQ_ERR_NULL;
+    if (!aligned(scales, 16) || !aligned(tiled, 16)) return MXQ_ERR_ALIGN;
+    const size_t col_tiles = (kblocks + 3) / 4, ntiles = ((rows + 127) / 128) * col_tiles;
+    const int grid = grid_for_tiles(ntiles, kThreads);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (kblocks % 4 == 0)
+        return launch_kernel(tile_scales_kernel<true>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
+    return launch_kernel(tile_scales_kernel<false>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
+}
 
 int mxq_quantize_tiled(const void* src, int src_dtype, size_t rows, size_t cols, int fmt, int block, void* codes,
                        uint8_t* tiled_scales, mxq_stream stream)
