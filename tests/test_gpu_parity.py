@@ -496,3 +496,66 @@ def test_dependent_chain_reusing_buffers_reads_fresh_data(nblk):
         got_c, got_v = kept[r]
         assert bits_equal(to_host(got_c.view(torch.uint8)), orc.pack(wc, 4)), (r, "codes")
         assert bits_equal(to_host(got_v), orc.fake_quant(want_v, "e2m3", mode=orc.FQ_DIRECT)), (r, "values")
+
+
+def test_randomized_cross_check_of_every_entry_point():
+    """Seeded random cases: block size, source type, length, magnitudes (zeros, outliers, a NaN or an
+    infinity now and then), tensors placed at 32-byte-aligned offsets inside larger buffers, a random
+    anchor-to-lower pair and a chained pair; every result against the oracle, bit for bit."""
+    rng = np.random.default_rng(20260411)
+    ints = ["int8", "int7", "int6", "int5", "int4", "int3", "int2"]
+    fps = ["e4m3", "e3m3", "e3m2", "e2m3", "e2m2", "e2m1"]
+
+    def place(x, pad):
+        if x.dtype == np.uint16:
+            buf = torch.zeros(x.size + 16 * pad + 64, dtype=torch.int16, device="cuda")
+            v = buf[16 * pad:16 * pad + x.size]
+            v.copy_(torch.from_numpy(x.view(np.int16)))
+            return v.view(torch.bfloat16)
+        buf = torch.zeros(x.size + 8 * pad + 64, dtype=torch.float32, device="cuda")
+        v = buf[8 * pad:8 * pad + x.size]
+        v.copy_(torch.from_numpy(x))
+        return v
+
+    for case in range(150):
+        block = int(rng.choice([16, 32, 32, 32, 64, 128]))
+        bf16 = bool(rng.random() < 0.6)
+        nblk = int(rng.choice([1, 2, 3, 5, 31, 33, 64, 127, 129, 257, 1000, 4097]))
+        if block == 16 and nblk % 2:
+            nblk += 1
+        x = rng.standard_normal((nblk, block)) * 2.0 ** rng.integers(-40, 40, (nblk, 1))
+        x[rng.random((nblk, block)) < 0.03] *= 64
+        x[rng.random((nblk, block)) < 0.05] = 0
+        x = x.astype(np.float32).reshape(-1)
+        if rng.random() < 0.15:
+            x[rng.integers(0, x.size)] = np.float32(rng.choice([np.inf, -np.inf, np.nan]))
+        if bf16:
+            x = inputs.to_bf16_bits(x)
+        n = x.size
+        xd = place(x, int(rng.integers(0, 4)))
+        fam = ints if rng.random() < 0.5 else fps
+        a, f = fam[0], str(rng.choice(fam))
+        what = (case, block, bf16, nblk, a, f)
+        ca, sa = mxq.quantize(xd, a, block)
+        oa, osa = orc.quantize(x, a, block)
+        assert bits_equal(to_host(ca), orc.pack(oa, 8)) and bits_equal(to_host(sa), osa), what
+        cf, sf = mxq.quantize(xd, f, block)
+        of, osf = orc.quantize(x, f, block)
+        assert bits_equal(to_host(cf), orc.pack(of, orc.bits(f))) and bits_equal(to_host(sf), osf), what
+        lc, ls = mxq.slice_scale(ca, sa, n, a, f, block)
+        wc, ws = orc.slice_scale(oa, osa, a, f, block)
+        assert bits_equal(to_host(lc), orc.pack(wc, orc.bits(f))) and bits_equal(to_host(ls), ws), what
+        g = str(rng.choice([h for h in fam[fam.index(f):] if orc.bits(h) <= orc.bits(f)]))
+        try:
+            w2, ws2 = orc.slice_scale(wc, ws, f, g, block)
+        except ValueError:
+            w2 = None                                          # not a legal pair (the exponent range would grow)
+        if w2 is not None:
+            cc, cs = mxq.slice_scale(lc, ls, n, f, g, block)
+            assert bits_equal(to_host(cc), orc.pack(w2, orc.bits(g))) and bits_equal(to_host(cs), ws2), what + (g,)
+        for dt, od in ((torch.float32, orc.F32), (torch.bfloat16, orc.BF16)):
+            v = mxq.dequantize(lc, ls, n, f, block, dtype=dt)
+            assert bits_equal(to_host(v), orc.dequantize(wc, ws, f, block, od)), what + (dt,)
+        for mode in (orc.FQ_DIRECT, orc.FQ_VIA_ANCHOR):
+            y = mxq.fake_quant(xd, f, block, mode)
+            assert bits_equal(to_host(y), orc.fake_quant(x, f, block, mode)), what + (mode,)
