@@ -242,3 +242,30 @@ def test_pack_layout(nb):
         assert packed[0] == (codes[0] | (codes[1] << 4))
     if nb == 8:
         assert np.array_equal(packed, codes)
+
+
+def test_ssmxint_other_tie_rules_would_differ_on_these_codes():
+    """What the reading of Eq. 4's Round is worth: how many of the 255 anchor codes would convert
+    differently under round-half-to-even or under round-half-up (toward +infinity), per exponent
+    difference.  Only exact ties differ -- 32 / 8 / 2 codes for ties-to-even (every second tie) and
+    31 / 7 / 1 for half-up (every negative tie that the clip does not absorb) -- so the oracle's rule
+    is pinned against both alternatives by those codes and by nothing else."""
+    for (src, dst), (want_even, want_up) in {("int8", "int6"): (32, 31), ("int8", "int4"): (8, 7),
+                                             ("int8", "int2"): (2, 1)}.items():
+        de = 8 - orc.bits(dst)
+        top = 2 ** (orc.bits(dst) - 1) - 1
+        even = up = 0
+        for p in range(-127, 128):
+            got = orc.slice_scale_elem(src, dst, p & 0xFF)
+            got = got - (1 << orc.bits(dst)) if got >> (orc.bits(dst) - 1) else got
+            x = Fraction(p, 1 << de)
+            lo = x.numerator // x.denominator
+            frac = x - lo
+            rne = lo + (1 if frac > Fraction(1, 2) or (frac == Fraction(1, 2) and lo % 2) else 0)
+            hup = (x + Fraction(1, 2)).numerator // (x + Fraction(1, 2)).denominator
+            clip = lambda q: max(-top, min(top, q))
+            even += clip(rne) != got
+            up += clip(hup) != got
+            if frac != Fraction(1, 2):
+                assert clip(rne) == got == clip(hup), (src, dst, p)
+        assert (even, up) == (want_even, want_up), (src, dst, even, up)
