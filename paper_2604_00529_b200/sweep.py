@@ -1,6 +1,6 @@
 """Bandwidth sweep of libmxq on one GPU.
 
-    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--all-formats] [--tiled] [--graph] [--json out.json]
+    python -m paper_2604_00529_b200.sweep [--min-log2 16] [--max-log2 31] [--model] [--all-formats] [--tiled] [--graph] [--warm] [--json out.json]
 
 `--graph` times CUDA-graph replays instead of direct launches.  For flat BF16 N(0,1) vectors of 2^k elements: direct quantization to each format, Slice-and-Scale
 for every anchor-to-lower pair, reconstruction and the fused fake-quant, timed with CUDA events over
@@ -33,6 +33,7 @@ def _peak():
         return 6650.0, "fallback"
 
 
+WARM = False      # --warm: one buffer set for every launch, so that sizes below the L2 capacity run out of L2
 GRAPH = False     # --graph: time the replay of a CUDA graph that holds the launches (no host cost per launch)
 
 
@@ -76,6 +77,8 @@ def sweep_size(n: int, base_dev: torch.Tensor, reps: int):
     copies = int(min(2048, max(2, -(-2 * L2_BYTES // (2 * n)))))
     if n * 2 * copies > 24 << 30:
         copies = 2
+    if WARM:
+        copies = 1
     xs = [base_dev[:n].clone() if n <= base_dev.numel() else base_dev.repeat(n // base_dev.numel()) for _ in range(copies)]
     u8 = dict(dtype=torch.uint8, device="cuda")
     out = {}
@@ -262,17 +265,21 @@ def main():
     ap.add_argument("--model", action="store_true")
     ap.add_argument("--all-formats", action="store_true", help="every element format of the paper at 2^26 elements")
     ap.add_argument("--tiled", action="store_true", help="tiled scale order at 8192 x 8192: fused against two passes")
+    ap.add_argument("--warm", action="store_true",
+                    help="reuse one buffer set for every launch (L2-resident figures for sizes that fit the 126 MB L2; "
+                         "the default rotates over enough copies to be cold)")
     ap.add_argument("--json", default=None)
     ap.add_argument("--graph", action="store_true",
                     help="capture each timed loop in a CUDA graph and time its replay: the figures then exclude the "
                          "host's cost of enqueuing a launch (about 8 us through this binding)")
     args = ap.parse_args()
-    global GRAPH
+    global GRAPH, WARM
     GRAPH = args.graph
+    WARM = args.warm
     mxq.load_library()
     peak, kind = _peak()
     base = torch.from_numpy(inputs.flat_bf16_normal(1 << 27, seed=5).view(np.int16)).cuda().view(torch.bfloat16)
-    result = {"peak_gbs": peak, "peak_kind": kind, "graph": GRAPH, "sizes": {}, "f32": {}, "model": {}}
+    result = {"peak_gbs": peak, "peak_kind": kind, "graph": GRAPH, "warm": WARM, "sizes": {}, "f32": {}, "model": {}}
     for k in range(args.min_log2, args.max_log2 + 1):
         n = 1 << k
         reps = 200 if k <= 22 else (50 if k <= 27 else 10)
