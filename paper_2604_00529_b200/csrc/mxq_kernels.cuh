@@ -1113,6 +1113,23 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                 if (sbk == 0xFFu) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+                } else if (F::id == MXQ_FP8_E4M3 && T::size == 2 &&
+                           !(has_e4m3_nan(w[u][(4 * K) % NWI]) | has_e4m3_nan(w[u][(4 * K + 1) % NWI]) |
+                             has_e4m3_nan(w[u][(4 * K + 2) % NWI]) | has_e4m3_nan(w[u][(4 * K + 3) % NWI]))) {
+                    // MXFP8 anchor codes (no NaN code among these 16): the widening conversion gives the
+                    // exact values, one FP32 multiply applies the scale as in the generic path below
+                    const float X = scale_value(sbk);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint32_t a, b;
+                        e4m3_word_to_f16(w[u][(4 * K + j) % NWI], a, b);
+                        float f0, f1, f2, f3;
+                        asm("{ .reg .b16 l, h; mov.b32 {l, h}, %4; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h;\n"
+                            "  mov.b32 {l, h}, %5; cvt.f32.f16 %2, l; cvt.f32.f16 %3, h; }"
+                            : "=f"(f0), "=f"(f1), "=f"(f2), "=f"(f3) : "r"(a), "r"(b));
+                        out[2 * j] = pack_bf16x2(f0 * X, f1 * X);
+                        out[2 * j + 1] = pack_bf16x2(f2 * X, f3 * X);
+                    }
                 } else {
                     const float X = scale_value(sbk);
                     static_for<EPS / 2>([&](auto i) {
