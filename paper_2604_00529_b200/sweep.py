@@ -135,6 +135,11 @@ def sweep_f32(n: int, reps: int):
         out["dequantize_%s_f32" % fmt] = (us, (1 + 1 / BLOCK + 4) * n / us / 1e3)
         us = _time(lambda j: mxq.fake_quant(xs[j], fmt, BLOCK, mxq.FQ_DIRECT, dst=ys[j]), copies, reps)
         out["fake_quant_f32_" + fmt] = (us, 8.0 * n / us / 1e3)
+    # the anchors reconstructed to BF16 (the 8-bit line of the algorithmic-bytes table)
+    yb = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+    for fmt in ("int8", "e4m3"):
+        us = _time(lambda j: mxq.dequantize(*cs[j], n, fmt, BLOCK, dst=yb[j]), copies, reps)
+        out["dequantize_%s_bf16" % fmt] = (us, (1 + 1 / BLOCK + 2) * n / us / 1e3)
     return out
 
 
@@ -291,7 +296,7 @@ def main():
         torch.cuda.empty_cache()
     f32 = sweep_f32(1 << 26, 50)
     result["f32"] = {name: {"us": round(us, 3), "gbs": round(g, 1)} for name, (us, g) in f32.items()}
-    print("FP32 entry points, 2^26 elements")
+    print("FP32 entry points and anchor reconstruction, 2^26 elements")
     for name, (us, g) in f32.items():
         print("  %-36s %10.2f us %8.1f GB/s  %5.1f %% of %s peak" % (name, us, g, 100 * g / peak, kind))
     if args.all_formats:
