@@ -17,7 +17,7 @@
  *     (src, dst, codes, out_codes, grad_*) must be 32-byte aligned (the kernels use 256-bit
  *     global accesses); scale buffers must be 16-byte aligned.  The library enqueues work on
  *     `stream` and returns without synchronising.  Unless an entry point says otherwise it
- *     allocates nothing.
+ *     allocates nothing and copies nothing (mxq_slice_scale_batched_static copies its item table).
  *   - Work goes to the CURRENT device, which must be the one the pointers belong to.  Kernels
  *     are launched with programmatic stream serialization allowed, so that a kernel's blocks
  *     can become resident while the previous kernel of the stream drains; each kernel waits
@@ -261,17 +261,25 @@ int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item *items, int count, int
  * The same conversion as mxq_slice_scale_batched for callers that cannot allocate device memory.
  * (The paper has no counterpart of this entry point; it exists for the library's users.)  Some
  * processes give all of HBM to a pool of their own at start-up, so a cudaMalloc made behind their
- * back fails or takes memory that was promised elsewhere; others run a loop where the host must
- * never stall, and cudaMalloc / cudaFree wait for the device.  For them the item table lives in a
+ * back fails or takes memory that was promised elsewhere; others run a loop that cannot take the
+ * device-wide synchronisation that cudaMalloc / cudaFree imply.  For them the item table lives in a
  * fixed array inside the library image: MXQ_STATIC_BATCH_MAX items and a small index, 57 KiB,
- * present on every GPU that loads libmxq until the process exits.  This call makes no cudaMalloc, cudaFree or other
- * allocating call, on the device or on the host heap, and converts up to MXQ_STATIC_BATCH_MAX
- * tensors in one launch.  (mxq_slice_scale_batched allocates nothing on the device either, but it
- * builds its launch tables on the host heap and needs one launch per 512 tensors.)
+ * present on every GPU that loads libmxq until the process exits.  The library makes no cudaMalloc,
+ * cudaFree or other allocating call here, on the device or on the host heap, and converts up to
+ * MXQ_STATIC_BATCH_MAX tensors in one launch.  (mxq_slice_scale_batched allocates nothing on the
+ * device either, but it builds its launch tables on the host heap and needs one launch per 512 tensors.)
+ * What the call does cost: it builds the table (57 KiB) on the caller's STACK, so a thread with a
+ * small stack needs about 64 KiB free; it copies the used part of it (0.6 - 57 KiB) to the device
+ * with a stream-ordered copy from that pageable memory, for which the CUDA runtime stages the bytes
+ * and may make the host wait for earlier work on `stream`; and the first call on a device may load
+ * the library's device code.  It is free of allocation, not free of host waits.
  *   - Arguments, checks and results are those of mxq_slice_scale_batched (block must be 32, 64 or
  *     128); in addition count > MXQ_STATIC_BATCH_MAX returns MXQ_ERR_SIZE and launches nothing.
  *   - The first call on each device looks up the array's device address (with that device current)
  *     and keeps it; make that first call before starting any stream capture.
+ *   - A call on a stream that is being captured returns MXQ_ERR_CUDA and enqueues nothing: the table
+ *     copy reads a buffer that no longer exists when the call has returned, so a recorded copy of it
+ *     would feed every replay stale stack bytes.
  *   - All calls on one device share the one table.  Each call rewrites the entries it uses and the
  *     kernel reads no others, so stale contents of an earlier call are harmless.  Calls ordered by
  *     one stream are safe; two calls whose work can overlap on the GPU (different streams, no

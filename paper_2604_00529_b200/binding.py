@@ -307,6 +307,63 @@ def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = Non
     return grad_in
 
 
+class PreparedCall:
+    """One C-ABI call with its arguments already marshalled, for buffers that persist (a model's
+    weights and their code buffers): ``prepare_*`` checks and converts the arguments once, calling the
+    object enqueues the operation on the current stream (or on ``stream``).  It keeps the tensors alive.
+    Per call this leaves the stream lookup and the foreign call itself (about 2 us instead of 5)."""
+
+    __slots__ = ("fn", "args", "what", "keep")
+
+    def __init__(self, fn, args, what, keep):
+        self.fn, self.args, self.what, self.keep = fn, args, what, keep
+
+    def __call__(self, stream=None) -> None:
+        rc = self.fn(*self.args, _stream(stream))
+        if rc != 0:
+            raise MxqError(rc, self.what)
+
+
+def prepare_quantize(src: torch.Tensor, fmt: str, block: int, codes: torch.Tensor, scales: torch.Tensor) -> PreparedCall:
+    """mxq_quantize(src -> codes, scales) as a PreparedCall."""
+    L = load_library()
+    return PreparedCall(L.mxq_quantize, (_dev(src, "src"), _dtype_id(src), src.numel(), FORMATS[fmt], block,
+                                         _dev(codes, "codes"), _dev(scales, "scales")), "mxq_quantize",
+                        (src, codes, scales))
+
+
+def prepare_slice_scale(codes: torch.Tensor, scales: torch.Tensor, n: int, src_fmt: str, dst_fmt: str, block: int,
+                        out_codes: torch.Tensor, out_scales: torch.Tensor) -> PreparedCall:
+    """mxq_slice_scale as a PreparedCall."""
+    L = load_library()
+    return PreparedCall(L.mxq_slice_scale, (_dev(codes, "codes"), _dev(scales, "scales"), n, block, FORMATS[src_fmt],
+                                            FORMATS[dst_fmt], _dev(out_codes, "out_codes"),
+                                            _dev(out_scales, "out_scales")), "mxq_slice_scale",
+                        (codes, scales, out_codes, out_scales))
+
+
+def prepare_dequantize(codes: torch.Tensor, scales: torch.Tensor, n: int, fmt: str, block: int,
+                       dst: torch.Tensor) -> PreparedCall:
+    """mxq_dequantize as a PreparedCall."""
+    L = load_library()
+    return PreparedCall(L.mxq_dequantize, (_dev(codes, "codes"), _dev(scales, "scales"), n, FORMATS[fmt], block,
+                                           _dev(dst, "dst"), _dtype_id(dst)), "mxq_dequantize", (codes, scales, dst))
+
+
+def prepare_fake_quant(src: torch.Tensor, fmt: str, block: int, mode: int, dst: torch.Tensor) -> PreparedCall:
+    """mxq_fake_quant as a PreparedCall."""
+    L = load_library()
+    return PreparedCall(L.mxq_fake_quant, (_dev(src, "src"), _dtype_id(src), src.numel(), FORMATS[fmt], block, mode,
+                                           _dev(dst, "dst")), "mxq_fake_quant", (src, dst))
+
+
+def prepare_fake_quant_bwd(grad_out: torch.Tensor, grad_in: torch.Tensor) -> PreparedCall:
+    """mxq_fake_quant_bwd as a PreparedCall."""
+    L = load_library()
+    return PreparedCall(L.mxq_fake_quant_bwd, (_dev(grad_out, "grad_out"), _dtype_id(grad_out), grad_out.numel(),
+                                               _dev(grad_in, "grad_in")), "mxq_fake_quant_bwd", (grad_out, grad_in))
+
+
 class _FakeQuantSTE(torch.autograd.Function):
     """Eq. 6 inside autograd: forward is mxq_fake_quant, backward the straight-through estimator."""
 

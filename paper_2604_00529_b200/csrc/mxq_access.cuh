@@ -161,24 +161,46 @@ __device__ __forceinline__ void store_bytes(void* p, const uint32_t (&w)[NW])
 // ---- staged tile stores ------------------------------------------------------------------------
 // A lane's piece of packed codes is OB bytes at lane * OB of its warp tile.  When OB is not one
 // aligned vector a direct store takes several narrow instructions, each of which touches every
-// 32-byte sector of the tile with a few bytes.  For the 7-bit formats that is seven 2- or 4-byte
-// stores per lane (measured 3.0 - 3.5 TB/s); their tiles go through shared memory instead: lanes
-// drop their pieces there and the warp copies the tile out as 16-byte pieces in address order
-// (5.4 TB/s).  With five or fewer direct stores (24, 20, 12, 10, 6 bytes) staging measured slower
-// than storing directly, so those keep the direct path.
+// 32-byte sector of the tile with a few bytes: a 6-bit tile (24 bytes per lane: a 16-byte and an
+// 8-byte store at a 24-byte stride) issues 2.9 times its sectors at L1, a 7-bit tile seven 2- or
+// 4-byte stores per lane.  Such tiles go through shared memory instead: lanes drop their pieces
+// there, and a whole tile leaves as ONE bulk copy shared -> global issued by one lane (the copy
+// engine writes full lines; no cluster, no tensor map, no multicast).  Only the ragged last tile of
+// a tensor is copied out by the lanes as 16-byte pieces.
+// Measured at 2^26 codes: MXINT8 -> MXINT6 and E4M3 -> E2M3 / E3M2 4 - 8 % faster than direct stores;
+// the 20-, 12- and 10-byte pieces of the 5- and 3-bit streams are faster stored directly (2 - 8 %).
 
 // store instructions a lane needs for a direct store of OB bytes
 __host__ __device__ constexpr int direct_store_count(int bytes) { return bytes / piece_align(bytes); }
 
 template <int OB>
 struct StagedTile {
-    static constexpr bool use = direct_store_count(OB) > 5;
+    static constexpr bool use = direct_store_count(OB) > 5 || OB == 24;
 };
 
-// Copy the first `nbytes` bytes of a warp's staging area to `gdst` (16-byte aligned, like the area).
+// Copy the first `nbytes` bytes of a warp's staging area to `gdst`; both are 16-byte aligned and
+// TILE_BYTES (a multiple of 16) is the size of a whole tile.  Every lane of the warp calls it, after
+// writing its own pieces to the area with ordinary stores.
+template <int TILE_BYTES>
 __device__ __forceinline__ void flush_stage(const uint8_t* stage, uint8_t* gdst, uint32_t nbytes)
 {
+    static_assert(TILE_BYTES % 16 == 0, "a bulk copy moves multiples of 16 bytes");
     const uint32_t lane = threadIdx.x & 31;
+    if (nbytes == TILE_BYTES) {
+        // the lanes' writes become visible to the copy engine, then one lane hands it the tile and
+        // waits until the engine has read the area (it may be rewritten or released afterwards)
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+            const uint32_t saddr = (uint32_t)__cvta_generic_to_shared(stage);
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         :: "l"(gdst), "r"(saddr), "r"(TILE_BYTES) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        }
+        __syncwarp();
+        return;
+    }
     __syncwarp();
     for (uint32_t i = lane * 16; i + 16 <= nbytes; i += 512)
         *reinterpret_cast<uint4*>(gdst + i) = *reinterpret_cast<const uint4*>(stage + i);

@@ -19,6 +19,7 @@
 // by byte permutes and one multiply, the sm_100a narrowing conversion instructions for MXFP.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <utility>
 #include <cuda_runtime.h>
 
@@ -154,21 +155,32 @@ __device__ __forceinline__ uint32_t group_max(uint32_t v)
 // Q_f: quantize (Eq. 1-3)
 // ------------------------------------------------------------------------------------------
 
-// 4 bytes holding 6-bit codes -> 24-bit stream c0 | c1 << 6 | c2 << 12 | c3 << 18
-__device__ __forceinline__ uint32_t squeeze6(uint32_t x)
+// Four 6-bit codes, one per byte, -> the 24-bit stream c0 | c1 << 6 | c2 << 12 | c3 << 18 in bits
+// 31..8 of the result (bits 7..0 clear).  Every field only ever moves LEFT relative to c3, so the
+// moves are multiply-adds (the multiply pipe) instead of shifts and selects on the logic pipe:
+// with the codes in bits 7..2 of their bytes, w + 3 (w & 0x00FF00FF) multiplies bytes 0 and 2 by 4,
+// which joins each byte pair into a 12-bit field (bits 15..4 and 31..20); y + 15 (y & 0xFFFF) then
+// multiplies the low field by 16, which joins the two.
+__device__ __forceinline__ uint32_t squeeze6_top(uint32_t w)           // codes in bits 7..2, bits 1..0 clear
 {
-    uint32_t y = (x & 0x003F003Fu) | ((x & 0x3F003F00u) >> 2);
-    return (y & 0x00000FFFu) | ((y >> 4) & 0x00FFF000u);
+    const uint32_t y = (w & 0x00FF00FFu) * 3u + w;
+    return (y & 0x0000FFFFu) * 15u + y;
 }
 
-// Four 24-bit streams -> three 32-bit words.  (Byte permutes would do the same job; shift + or
-// measured 5 % faster on the MXINT8 -> MXINT6 conversion, where the logic pipe is the bound.)
+__device__ __forceinline__ uint32_t squeeze6_low(uint32_t w)           // codes in bits 5..0, bits 7..6 clear
+{
+    const uint32_t y = (w & 0x00FF00FFu) * 12u + w * 4u;
+    return (y & 0x0000FFFFu) * 15u + y;
+}
+
+// Four such streams (each in bits 31..8 of its word) -> three 32-bit words: whole bytes, so three
+// byte permutes.
 __device__ __forceinline__ void join24(uint32_t z0, uint32_t z1, uint32_t z2, uint32_t z3, uint32_t& o0, uint32_t& o1,
                                        uint32_t& o2)
 {
-    o0 = z0 | (z1 << 24);
-    o1 = (z1 >> 8) | (z2 << 16);
-    o2 = (z2 >> 16) | (z3 << 8);
+    o0 = __byte_perm(z0, z1, 0x5321);
+    o1 = __byte_perm(z1, z2, 0x6532);
+    o2 = __byte_perm(z2, z3, 0x7653);
 }
 
 // Four B-bit codes, one per byte with the upper bits clear, -> one 4B-bit value (c0 | c1 << B | ...).
@@ -268,8 +280,8 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
         } else if constexpr (F::bits == 6 && NQ % 4 == 0) {
 #pragma unroll
             for (int g = 0; g < NQ / 4; ++g) {
-                const uint32_t s0 = squeeze6(z[4 * g]), s1 = squeeze6(z[4 * g + 1]), s2 = squeeze6(z[4 * g + 2]),
-                               s3 = squeeze6(z[4 * g + 3]);
+                const uint32_t s0 = squeeze6_low(z[4 * g]), s1 = squeeze6_low(z[4 * g + 1]), s2 = squeeze6_low(z[4 * g + 2]),
+                               s3 = squeeze6_low(z[4 * g + 3]);
                 join24(s0, s1, s2, s3, out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
             }
         } else {
@@ -318,7 +330,7 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
     const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
     uint8_t* stage = nullptr;
     if constexpr (StagedTile<OB>::use) {
-        __shared__ __align__(16) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
+        __shared__ __align__(128) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
         stage = stage_area + (threadIdx.x >> 5) * (32 * U * OB);
     }
 
@@ -355,7 +367,7 @@ quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restr
         }
         if constexpr (StagedTile<OB>::use) {
             const size_t first = tile * (32 * U), left = nunits - first;
-            flush_stage(stage, codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
+            flush_stage<32 * U * OB>(stage, codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
         }
     }
 }
@@ -600,26 +612,42 @@ fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count,
 // ------------------------------------------------------------------------------------------
 
 // Eq. 4 on four MXINT8 codes at once (one per byte): returns the four low-format codes, one per
-// byte, in the low BL bits.  Sign-magnitude SWAR; no carry ever crosses a byte.  The integer/logic
-// pipe is the scarce resource here, so the two places that need the per-byte sign as a 0/1 value
-// take it from the 0xFF/0x00 mask by one multiply-add with 255^-1 (mod 2^32), which runs on the
-// multiply pipe: mask = 255 * sum(s_i 256^i), hence mask * 255^-1 = sum(s_i 256^i) exactly.
+// byte, in the TOP BL bits of the byte (the bits below are clear).  Sign-magnitude SWAR; no carry
+// crosses a byte until the last step, whose stray carry lands in a bit that is masked off.
+//   full : 0xFF in the bytes that are negative (byte permute with sign replication)
+//   a    : |p| - s per byte, s the 0/1 sign (one's complement of the negative bytes)
+//   T    : |p| + 2^(de-1) <= 128 + 2^(de-1); the shifted value q = T >> de sits in T's top BL bits.
+//          q reaches 2^(BL-1) exactly when T >= 128, and then those top bits read 100..0: flipping
+//          them (xor with the replicated top bit of T) gives 011..1, the clipped magnitude.
+//   two's complement of the negative bytes: flip the BL bits, add one at bit de.  The add can carry
+//   out of a byte only for q = 0 (the bits are all ones), into bit 0 of the next byte, which is
+//   cleared before (so that it cannot travel) and after.
+// The integer/logic pipe is the scarce resource here, so the per-byte 0/1 sign comes from the
+// 0xFF/0x00 mask by a multiply-add with 255^-1 (mod 2^32), which runs on the multiply pipe:
+// mask = 255 * sum(s_i 256^i), hence mask * 255^-1 = sum(s_i 256^i) exactly.
+// (Checked against the scalar definition for all 2^32 input words on the host.)
 template <int BL>
-__device__ __forceinline__ uint32_t ss_int8_word(uint32_t x)
+__device__ __forceinline__ uint32_t ss_int8_word_top(uint32_t x)
 {
     constexpr int de = 8 - BL;
     constexpr uint32_t k01 = 0x01010101u;
     constexpr uint32_t kInv255 = 0xFEFEFEFFu;
     constexpr uint32_t kH = k01 * (1u << (de - 1));            // rounding increment
-    constexpr uint32_t kLow = k01 * (0xFFu >> de);
-    constexpr uint32_t kMask = k01 * ((1u << BL) - 1u);
-    uint32_t full;                                            // 0xFF in the bytes that are negative
-    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(x));  // selector bit 3: replicate the byte's sign
-    const uint32_t a = x ^ full;                               // |p| - s
-    const uint32_t t = a + full * kInv255 + kH;                // |p| + 2^(de-1) <= 127 + 64
-    const uint32_t c = (t >> 7) & k01;                         // 1 where the shifted value would be 2^(BL-1)
-    const uint32_t q = ((t >> de) & kLow) - c;                 // clipped to 2^(BL-1) - 1
-    return (full * kInv255 + (q ^ (full & kMask))) & kMask;    // two's complement in BL bits
+    constexpr uint32_t kTop = k01 * ((0xFFu << de) & 0xFFu);   // the top BL bits of every byte
+    uint32_t full, ov;
+    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(full) : "r"(x)); // selector bit 3: replicate the byte's sign
+    const uint32_t a = x ^ full;
+    const uint32_t t = a + (full * kInv255 + kH);
+    asm("prmt.b32 %0, %1, %1, 0xBA98;" : "=r"(ov) : "r"(t));   // 0xFF where the magnitude clips
+    const uint32_t m = (t ^ ov ^ full) & kTop;
+    return (full * (kInv255 << de) + m) & kTop;
+}
+
+// The same four codes in the low BL bits of their bytes.
+template <int BL>
+__device__ __forceinline__ uint32_t ss_int8_word(uint32_t x)
+{
+    return ss_int8_word_top<BL>(x) >> (8 - BL);
 }
 
 __device__ __forceinline__ bool has_e4m3_nan(uint32_t x)
@@ -750,7 +778,7 @@ __device__ __forceinline__ void ss_e4m3_unit_fast(const uint32_t (&in)[8], uint3
     } else if constexpr (FL::hw_cvt) {
         uint32_t z[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) z[j] = squeeze6(ss_e4m3_word_to6<FL>(in[j]));
+        for (int j = 0; j < 8; ++j) z[j] = squeeze6_low(ss_e4m3_word_to6<FL>(in[j]));
 #pragma unroll
         for (int g = 0; g < 2; ++g)
             join24(z[4 * g + 0], z[4 * g + 1], z[4 * g + 2], z[4 * g + 3], out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
@@ -770,17 +798,17 @@ __device__ __forceinline__ void slice_scale_unit(const uint32_t (&in)[NWI], uint
 #pragma unroll
         for (int j = 0; j < NWO; ++j) out[j] = in[j];
     } else if constexpr (FH::id == MXQ_INT8 && FL::bits == 4) {
-        // even / odd codes of 8 -> low / high nibbles of 4 bytes
+        // the codes come back in the high nibbles: w * 17 drops each one into the low nibble of the
+        // byte above as well, so bytes 1 and 3 of it hold c0 | c1 << 4 and c2 | c3 << 4
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            uint32_t e = __byte_perm(in[2 * j], in[2 * j + 1], 0x6420);
-            uint32_t o = __byte_perm(in[2 * j], in[2 * j + 1], 0x7531);
-            out[j] = ss_int8_word<4>(e) | (ss_int8_word<4>(o) << 4);
+            const uint32_t a = ss_int8_word_top<4>(in[2 * j]), b = ss_int8_word_top<4>(in[2 * j + 1]);
+            out[j] = __byte_perm(a * 16u + a, b * 16u + b, 0x7531);
         }
     } else if constexpr (FH::id == MXQ_INT8 && FL::bits == 6) {
         uint32_t z[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) z[j] = squeeze6(ss_int8_word<6>(in[j]));
+        for (int j = 0; j < 8; ++j) z[j] = squeeze6_top(ss_int8_word_top<6>(in[j]));
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
             join24(z[4 * g + 0], z[4 * g + 1], z[4 * g + 2], z[4 * g + 3], out[3 * g + 0], out[3 * g + 1], out[3 * g + 2]);
@@ -840,7 +868,7 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
     }
     if constexpr (StagedTile<OB>::use) {
         const size_t first = tile * (32 * U), left = nunits - first;
-        flush_stage(stage, out_codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
+        flush_stage<32 * U * OB>(stage, out_codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
     }
     if (nscales > nunits) {
 #pragma unroll
@@ -858,15 +886,27 @@ __device__ __forceinline__ uint8_t* slice_scale_stage()
 {
     constexpr int OB = 4 * FL::bits;
     if constexpr (StagedTile<OB>::use) {
-        __shared__ __align__(16) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
+        __shared__ __align__(128) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
         return stage_area + (threadIdx.x >> 5) * (32 * U * OB);
     } else {
         return nullptr;
     }
 }
 
+// Resident CTAs (of 128 threads) per SM the single-tensor kernel is compiled for, i.e. its register
+// budget.  Measured at 2^26 codes with 10 / 12 / 14 / 16 CTAs: the MXINT conversions are fastest with
+// room for 40 - 48 registers (both lane units' arithmetic interleaves; MXINT8 -> MXINT4 8 % faster
+// than at 32 registers), the MXFP ones with 14 - 16 CTAs (E4M3 -> E2M3 8 % faster than at 50
+// registers); with tiled scale outputs 14 CTAs would spill, so those keep 12.
+template <class FH, class SCALES>
+__host__ __device__ constexpr int slice_scale_min_ctas()
+{
+    if constexpr (!std::is_same_v<SCALES, uint8_t*>) return 12;
+    else return FH::kind == KIND_INT ? 10 : 14;
+}
+
 template <class FH, class FL, int U, int THREADS, class SCALES = uint8_t*>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, slice_scale_min_ctas<FH, SCALES>())
 slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                    size_t nscales, uint8_t* __restrict__ out_codes, SCALES out_scales)
 {
@@ -898,11 +938,11 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
     uint8_t* stage1 = nullptr;
     uint8_t* stage2 = nullptr;
     if constexpr (StagedTile<OB1>::use) {
-        __shared__ __align__(16) uint8_t area1[(THREADS / 32) * 32 * U * OB1];
+        __shared__ __align__(128) uint8_t area1[(THREADS / 32) * 32 * U * OB1];
         stage1 = area1 + (threadIdx.x >> 5) * (32 * U * OB1);
     }
     if constexpr (StagedTile<OB2>::use) {
-        __shared__ __align__(16) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
+        __shared__ __align__(128) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
         stage2 = area2 + (threadIdx.x >> 5) * (32 * U * OB2);
     }
     prefetch_tile<U, IB>(codes, tile, nunits);
@@ -950,8 +990,8 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
     {
         const size_t first = tile * (32 * U), left = nunits - first;
         const uint32_t valid = (uint32_t)(left < 32 * U ? left : 32 * U);
-        if constexpr (StagedTile<OB1>::use) flush_stage(stage1, out_codes1 + first * OB1, valid * OB1);
-        if constexpr (StagedTile<OB2>::use) flush_stage(stage2, out_codes2 + first * OB2, valid * OB2);
+        if constexpr (StagedTile<OB1>::use) flush_stage<32 * U * OB1>(stage1, out_codes1 + first * OB1, valid * OB1);
+        if constexpr (StagedTile<OB2>::use) flush_stage<32 * U * OB2>(stage2, out_codes2 + first * OB2, valid * OB2);
     }
     if (nscales > nunits) {
 #pragma unroll

@@ -4,7 +4,11 @@
 //
 // Who needs this: a serving process that has handed the whole HBM to its own pool (weights, KV
 // cache) so that a stray cudaMalloc fails or eats into a budget somebody else planned; and a
-// latency-critical loop, where cudaMalloc / cudaFree stall the host until the device is idle.
+// loop that must not take the device-wide synchronisation cudaMalloc / cudaFree imply.
+// What the call still costs: a 57 KiB table on the caller's stack (a thread with a small stack
+// needs about 64 KiB free), a stream-ordered copy of 0.6 - 57 KiB from that pageable table, for
+// which the runtime may make the host wait on the stream, and on the first call per device the
+// lookup of the array's address (which can load the library's device code).
 #include <cstddef>
 #include <mutex>
 
@@ -92,15 +96,29 @@ extern "C" int mxq_slice_scale_batched_static(const mxq_ss_item* items, int coun
     }
     if (used == 0) return MXQ_OK;
 
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The table copy below reads `staged`, which is gone when this function returns.  A stream that is
+    // being captured would record the copy instead of performing it, and every later replay would read
+    // a dead stack frame and hand the kernel garbage pointers: refuse before anything is enqueued.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    if (capturing != cudaStreamCaptureStatusNone) return MXQ_ERR_CUDA;
+
     build_tile_index(staged.index, host, used, tiles);
     StaticTable* table = nullptr;
     if (int rc = static_table(&table)) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     // Entries [0, used) are rewritten by every call and the kernel reads no others, so nothing in
     // the table has to start from zero.  The source is pageable stack memory: the runtime has
-    // staged the bytes by the time this returns.
+    // staged the bytes by the time this returns (it may make the host wait for earlier work of the
+    // stream to do so).
     const size_t nbytes = offsetof(StaticTable, items) + sizeof(SsDeviceItem) * (size_t)used;
-    if (cudaMemcpyAsync(table, &staged, nbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return MXQ_ERR_CUDA;
+    if (cudaMemcpyAsync(table, &staged, nbytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
     return launch_slice_scale_batched(table->items, &table->index, used, tiles, src_fmt, dst_fmt, s);
 }
 #pragma GCC visibility pop

@@ -13,13 +13,23 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
-    """GPU tests are skipped (not failed) where no device exists and -m gpu was not asked for."""
+    """Without a CUDA device the GPU tests are skipped -- unless the run asked for them (`-m gpu`):
+    then they stay in and fail, so that a GPU run on a box whose CUDA context did not come up cannot
+    pass with every parity test skipped."""
     try:
         import torch
         has_gpu = torch.cuda.is_available()
     except Exception:  # pragma: no cover
         has_gpu = False
     if has_gpu:
+        return
+    asked = (config.getoption("-m") or "").replace(" ", "")
+    if "gpu" in asked and "notgpu" not in asked:
+        def no_device():
+            pytest.fail("this run selected the GPU tests (-m gpu) but no CUDA device is available")
+        for item in items:
+            if "gpu" in item.keywords:
+                item.obj = no_device            # fail, do not skip
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for item in items:
