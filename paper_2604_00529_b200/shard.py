@@ -39,3 +39,29 @@ def output_ranges(lo: int, hi: int, bits: int, block: int):
     """Byte ranges ((codes_lo, codes_hi), (scales_lo, scales_hi)) of the packed outputs that the
     element range [lo, hi) owns."""
     return (lo * bits // 8, hi * bits // 8), (lo // block, hi // block)
+
+
+def quantize_shard(src, fmt: str, block: int, codes, scales, rank: int, world: int, stream=None):
+    """Rank `rank`'s part of mxq_quantize(src -> codes, scales): converts the rank's run of whole blocks
+    of the full tensor `src` into the matching byte ranges of the full output buffers (all of them
+    device tensors of the FULL size; with one process per GPU each rank passes its own copies or
+    views).  Returns the element range [lo, hi) it converted."""
+    from . import binding
+    lo, hi = block_range(src.numel(), block, rank, world)
+    if hi > lo:
+        (c_lo, c_hi), (s_lo, s_hi) = output_ranges(lo, hi, binding.format_bits(fmt), block)
+        binding.quantize(src.reshape(-1)[lo:hi], fmt, block, codes[c_lo:c_hi], scales[s_lo:s_hi], stream)
+    return lo, hi
+
+
+def slice_scale_shard(codes, scales, n: int, src_fmt: str, dst_fmt: str, block: int, out_codes, out_scales,
+                      rank: int, world: int, stream=None):
+    """Rank `rank`'s part of mxq_slice_scale over full-size buffers (see quantize_shard)."""
+    from . import binding
+    lo, hi = block_range(n, block, rank, world)
+    if hi > lo:
+        (a_lo, a_hi), (s_lo, s_hi) = output_ranges(lo, hi, binding.format_bits(src_fmt), block)
+        (c_lo, c_hi), _ = output_ranges(lo, hi, binding.format_bits(dst_fmt), block)
+        binding.slice_scale(codes[a_lo:a_hi], scales[s_lo:s_hi], hi - lo, src_fmt, dst_fmt, block,
+                            out_codes[c_lo:c_hi], out_scales[s_lo:s_hi], stream)
+    return lo, hi

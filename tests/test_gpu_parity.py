@@ -384,6 +384,67 @@ def test_quantize_then_dequantize_equals_fake_quant(fmt):
     assert bits_equal(v, gpu_fake_quant(x, fmt))
 
 
+@pytest.mark.parametrize("world", [2, 3, 8])
+def test_sharded_conversion_stitches_to_the_unsharded_one(world):
+    """The multi-GPU path: every rank converts its own run of whole blocks into its own byte range of
+    the full outputs, with no exchange.  The ranks run here one after another on one GPU (independent
+    launches that do not wait on one another); the stitched result must be the oracle's whole-tensor
+    result, byte for byte, and nothing outside a rank's range may be touched by it."""
+    from paper_2604_00529_b200.shard import block_range, quantize_shard, slice_scale_shard
+    nblk = 5003                                          # 157 chunks of 32 blocks: a ragged split for every world size
+    x = _mixed_f32(nblk, seed=77)
+    n = x.size
+    xd = to_dev(x)
+    codes, scales = Guarded(n), Guarded(n // 32)
+    lc, ls = Guarded(n // 2), Guarded(n // 32)
+    covered = 0
+    for rank in range(world):
+        lo, hi = quantize_shard(xd, "int8", 32, codes.view, scales.view, rank, world)
+        assert (lo, hi) == block_range(n, 32, rank, world) and lo == covered
+        covered = hi
+        torch.cuda.synchronize()
+        got = to_host(codes.view)
+        assert np.all(got[hi:] == 0xA5), "rank %d wrote beyond its range" % rank
+    assert covered == n
+    for rank in reversed(range(world)):                  # any order: the shards are independent
+        slice_scale_shard(codes.view, scales.view, n, "int8", "int4", 32, lc.view, ls.view, rank, world)
+    torch.cuda.synchronize()
+    for g in (codes, scales, lc, ls):
+        g.check()
+    wc, ws = orc.quantize(x, "int8")
+    assert bits_equal(to_host(codes.view), orc.pack(wc, 8)) and bits_equal(to_host(scales.view), ws)
+    w4, s4 = orc.slice_scale(wc, ws, "int8", "int4")
+    assert bits_equal(to_host(lc.view), orc.pack(w4, 4)), first_diff(to_host(lc.view), orc.pack(w4, 4))
+    assert bits_equal(to_host(ls.view), s4)
+
+
+def test_prepared_calls_give_the_same_bytes():
+    """The pre-marshalled call objects of the binding enqueue the same operations as the plain functions."""
+    x = _mixed_f32(700, seed=5)
+    n = x.size
+    xd = to_dev(x)
+    c, s = Guarded(n), Guarded(n // 32)
+    lc, ls = Guarded(n * 6 // 8), Guarded(n // 32)
+    y, f, g = Guarded(4 * n, torch.float32), Guarded(4 * n, torch.float32), Guarded(4 * n, torch.float32)
+    calls = [mxq.prepare_quantize(xd, "e4m3", 32, c.view, s.view),
+             mxq.prepare_slice_scale(c.view, s.view, n, "e4m3", "e2m3", 32, lc.view, ls.view),
+             mxq.prepare_dequantize(lc.view, ls.view, n, "e2m3", 32, y.view),
+             mxq.prepare_fake_quant(xd, "e2m3", 32, mxq.FQ_VIA_ANCHOR, f.view),
+             mxq.prepare_fake_quant_bwd(f.view, g.view)]
+    for _ in range(2):                                   # a prepared call may be used any number of times
+        for call in calls:
+            call()
+    torch.cuda.synchronize()
+    for buf in (c, s, lc, ls, y, f, g):
+        buf.check()
+    wc, ws = orc.quantize(x, "e4m3")
+    w6, s6 = orc.slice_scale(wc, ws, "e4m3", "e2m3")
+    assert bits_equal(to_host(c.view), orc.pack(wc, 8)) and bits_equal(to_host(s.view), ws)
+    assert bits_equal(to_host(lc.view), orc.pack(w6, 6)) and bits_equal(to_host(ls.view), s6)
+    want = orc.dequantize(w6, s6, "e2m3")
+    assert bits_equal(to_host(y.view), want) and bits_equal(to_host(f.view), want) and bits_equal(to_host(g.view), want)
+
+
 def test_smallest_and_empty_inputs():
     x = np.array([1.0] + [0.25] * 31, np.float32)
     c, s = gpu_quantize(x, "int8")

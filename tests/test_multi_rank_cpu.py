@@ -83,3 +83,30 @@ def test_block_ranges_cover_and_align(world, nblk):
         assert hi == lo or lo % (32 * 32) == 0      # a rank with work starts on an aligned chunk
         prev = hi
     assert prev == n
+
+
+def test_bench_gpus_flag_starts_the_ranks():
+    """`bench.py --gpus 2` outside torchrun starts two ranks itself (here the CPU self-test worker over
+    gloo) and rank 0 prints one line with n_gpus = 2 and the max over the ranks."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "selftest"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["max_over_ranks"] == 2.0
+
+
+def test_bench_under_a_launcher_reads_the_rank_environment():
+    """Started by a launcher (WORLD_SIZE set), bench.py is one rank and starts nothing itself: a
+    one-rank environment prints n_gpus = 1 even with --gpus 1."""
+    import json
+    import subprocess
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "1", "--impl", "selftest"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr
+    assert json.loads(out.stdout.strip().splitlines()[-1])["n_gpus"] == 1
