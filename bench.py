@@ -7,8 +7,8 @@ One invocation times all five workloads of the method and prints ONE JSON line o
 
 Headline (`value`, `config.workload`): the whole-model workload -- the 224 BF16 linear weights of an 8B
 Llama-shaped decoder (6.98 G elements).  A *step* is one pass of the whole hot path over that weight
-set: quantize every tensor to the MXINT8 and the MXFP8 (E4M3) anchor (Eq. 1-3), Slice-and-Scale both
-anchors to MXINT6 / MXINT4 and MXFP6 (E2M3) / MXFP4 (E2M1) with one batched launch per target (Eq. 4-5,
+set, ten launches that each cover all 224 tensors: quantize to the MXINT8 and the MXFP8 (E4M3) anchor (Eq. 1-3), Slice-and-Scale both
+anchors to MXINT6 / MXINT4 and MXFP6 (E2M3) / MXFP4 (E2M1) (Eq. 4-5,
 the on-the-fly conversion of Sec. 3.5), reconstruct the two 4-bit sets to BF16, run the fused fake-quant
 of all weights through the anchor (Eq. 6) and its straight-through backward.  180 GB of algorithmic
 traffic per step, every buffer far larger than L2.  K steps run back to back between two CUDA events;
@@ -70,14 +70,14 @@ def b_dequantize(fmt: str, dst_bytes: int) -> float:
 
 # the op groups of the headline step, in order, with their algorithmic bytes per element
 STEP_OPS = [
-    ("quantize_bf16_int8", b_quantize(2, "int8")),
-    ("quantize_bf16_e4m3", b_quantize(2, "e4m3")),
+    ("quantize_batched_bf16_int8", b_quantize(2, "int8")),
+    ("quantize_batched_bf16_e4m3", b_quantize(2, "e4m3")),
     ("ss_batched_int8_int6", b_slice_scale("int6")),
     ("ss_batched_int8_int4", b_slice_scale("int4")),
     ("ss_batched_e4m3_e2m3", b_slice_scale("e2m3")),
     ("ss_batched_e4m3_e2m1", b_slice_scale("e2m1")),
-    ("dequantize_int4_bf16", b_dequantize("int4", 2)),
-    ("dequantize_e2m1_bf16", b_dequantize("e2m1", 2)),
+    ("dequantize_batched_int4_bf16", b_dequantize("int4", 2)),
+    ("dequantize_batched_e2m1_bf16", b_dequantize("e2m1", 2)),
     ("fake_quant_batched_bf16_e2m3_via_anchor", 4.0),
     ("fake_quant_bwd_bf16", 4.0),
 ]
@@ -107,7 +107,7 @@ def kernel_sources_digest() -> str:
     d = os.path.join(ROOT, "paper_2604_00529_b200", "csrc")
     h = hashlib.sha256()
     for name in sorted(os.listdir(d)):
-        if name.endswith((".cu", ".cuh", ".h")):
+        if name.startswith("mxq_") and name.endswith((".cu", ".cuh", ".h")):
             h.update(name.encode())
             h.update(open(os.path.join(d, name), "rb").read())
     return h.hexdigest()[:16]
@@ -566,6 +566,8 @@ class WholeModel:
         self.q_calls = {f: [mxq.prepare_quantize(self.w[int(offs[k]):int(offs[k + 1])], f, BLOCK,
                                                  view(self.anchor[f][0], k), sview(self.anchor[f][1], k)) for k in T]
                         for f in ("int8", "e4m3")}
+        self.q_tables = {f: mxq.make_q_items([(self.w[int(offs[k]):int(offs[k + 1])], view(self.anchor[f][0], k),
+                                               sview(self.anchor[f][1], k)) for k in T]) for f in ("int8", "e4m3")}
         self.ss_pairs = (("int8", "int6"), ("int8", "int4"), ("e4m3", "e2m3"), ("e4m3", "e2m1"))
         self.ss_items = {}
         self.ss_calls = {}
@@ -577,24 +579,27 @@ class WholeModel:
         self.dq_calls = {t: [mxq.prepare_dequantize(view(self.target[t][0], k, BITS[t]), sview(self.target[t][1], k),
                                                     self.sizes[k], t, BLOCK, self.deq[int(offs[k]):int(offs[k + 1])]) for k in T]
                          for t in ("int4", "e2m1")}
+        self.dq_tables = {t: mxq.make_dq_items([(view(self.target[t][0], k, BITS[t]), sview(self.target[t][1], k),
+                                                 self.sizes[k], self.deq[int(offs[k]):int(offs[k + 1])]) for k in T])
+                          for t in ("int4", "e2m1")}
         self.fq_pairs = [(self.w[int(offs[k]):int(offs[k + 1])], self.fq[int(offs[k]):int(offs[k + 1])]) for k in T]
         self.fq_table = mxq.make_fq_items(self.fq_pairs)
         self.bwd = mxq.prepare_fake_quant_bwd(self.fq, self.grad)
-        self.launches_per_step = 2 * len(self.sizes) + 4 + 2 * len(self.sizes) + 1 + 1
+        self.launches_per_step = len(STEP_OPS)               # every op group is one launch over the 224 tensors
 
     def step(self, mark=None):
         """One pass of the whole hot path over the weight set; `mark(k)` is called before op group k
         (the order of STEP_OPS) and after the last one."""
         mxq = self.mxq
         groups = [
-            lambda: [c() for c in self.q_calls["int8"]],
-            lambda: [c() for c in self.q_calls["e4m3"]],
+            lambda: mxq.quantize_batched(self.q_tables["int8"], "int8", BLOCK),
+            lambda: mxq.quantize_batched(self.q_tables["e4m3"], "e4m3", BLOCK),
             lambda: mxq.slice_scale_batched(self.ss_items[("int8", "int6")], "int8", "int6", BLOCK),
             lambda: mxq.slice_scale_batched(self.ss_items[("int8", "int4")], "int8", "int4", BLOCK),
             lambda: mxq.slice_scale_batched(self.ss_items[("e4m3", "e2m3")], "e4m3", "e2m3", BLOCK),
             lambda: mxq.slice_scale_batched(self.ss_items[("e4m3", "e2m1")], "e4m3", "e2m1", BLOCK),
-            lambda: [c() for c in self.dq_calls["int4"]],
-            lambda: [c() for c in self.dq_calls["e2m1"]],
+            lambda: mxq.dequantize_batched(self.dq_tables["int4"], "int4", BLOCK),
+            lambda: mxq.dequantize_batched(self.dq_tables["e2m1"], "e2m1", BLOCK),
             lambda: mxq.fake_quant_batched(self.fq_table, "e2m3", BLOCK, mxq.FQ_VIA_ANCHOR),
             lambda: self.bwd(),
         ]
@@ -617,6 +622,20 @@ def whole_model_conversions(bench: Bench, wm: WholeModel):
         tp = bench.regions(lambda j: [c() for c in wm.ss_calls[(a, t)]], 1, reps=1, warm=1)
         out["%s_to_%s" % (a, t)] = {"batched_one_launch": bench.record(tb, nbytes, wm.total),
                                     "per_tensor_launches": bench.record(tp, nbytes, wm.total, launches_per_call=len(wm.sizes))}
+        bench.launches += (REGIONS + 1) * (1 + len(wm.sizes))
+    for f in ("int8", "e4m3"):
+        nbytes = b_quantize(2, f) * wm.total
+        tb = bench.regions(lambda j: mxq.quantize_batched(wm.q_tables[f], f, BLOCK), 1, reps=1, warm=1)
+        tp = bench.regions(lambda j: [c() for c in wm.q_calls[f]], 1, reps=1, warm=1)
+        out["quantize_bf16_%s" % f] = {"batched_one_launch": bench.record(tb, nbytes, wm.total),
+                                       "per_tensor_launches": bench.record(tp, nbytes, wm.total, launches_per_call=len(wm.sizes))}
+        bench.launches += (REGIONS + 1) * (1 + len(wm.sizes))
+    for t in ("int4", "e2m1"):
+        nbytes = b_dequantize(t, 2) * wm.total
+        tb = bench.regions(lambda j: mxq.dequantize_batched(wm.dq_tables[t], t, BLOCK), 1, reps=1, warm=1)
+        tp = bench.regions(lambda j: [c() for c in wm.dq_calls[t]], 1, reps=1, warm=1)
+        out["dequantize_%s_bf16" % t] = {"batched_one_launch": bench.record(tb, nbytes, wm.total),
+                                         "per_tensor_launches": bench.record(tp, nbytes, wm.total, launches_per_call=len(wm.sizes))}
         bench.launches += (REGIONS + 1) * (1 + len(wm.sizes))
     for fmt in ("e2m3", "int4"):
         tb = bench.regions(lambda j: mxq.fake_quant_batched(wm.fq_table, fmt, BLOCK, mxq.FQ_VIA_ANCHOR), 1, reps=1, warm=1)
@@ -867,12 +886,11 @@ def run_cuda(args):
         per_op[name] = {"ms": round(med, 4), "ms_min": round(min(ms), 4), "ms_max": round(max(ms), 4),
                         "gbs": round(gbs, 1), "gelem_s": round(total_elems / (med * 1e-3) / 1e9, 2),
                         "frac_of_%s_peak" % peak_kind: round(gbs / peak, 4), "frac_of_8000": round(gbs / 8000.0, 4),
-                        "launches": n_tensors if name.startswith(("quantize", "dequantize")) else 1}
+                        "launches": 1}
         if mhz:
             per_op[name]["ms_x_ghz"] = round(med * mhz / 1e3, 4)
-    # the dominant kernel: the single launch that takes the longest (the batched fake-quant or the copy)
-    single = [k for k, (name, _) in enumerate(STEP_OPS) if per_op[name]["launches"] == 1]
-    top = max(single, key=lambda k: statistics.median(op_ms[k]))
+    # the dominant kernel: the launch that takes the longest (the batched fake-quant or the copy)
+    top = max(range(nops), key=lambda k: statistics.median(op_ms[k]))
     top_name, top_bpe = STEP_OPS[top]
     top_ms = sum(op_ms[top]) / K                              # average launch duration over the timed region
     top_gbs = top_bpe * total_elems / (top_ms * 1e-3) / 1e9
@@ -925,7 +943,7 @@ def run_ncu_case(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     u8 = dict(dtype=torch.uint8, device=dev)
-    n_ss, n = 1 << 30, 1 << 29
+    n_ss, n = 1 << args.case_log2, 1 << (args.case_log2 - 1)
     x = torch.from_numpy(inputs.flat_bf16_normal(1 << 24, seed=5).view(np.int16)).to(dev).view(torch.bfloat16).repeat(n >> 24)
     codes, scales = torch.empty(n_ss, **u8), torch.empty(n_ss // BLOCK, **u8)
     out_c, out_s = torch.empty(n_ss * 6 // 8, **u8), torch.empty(n_ss // BLOCK, **u8)
@@ -949,8 +967,10 @@ def run_ncu_case(args):
         mxq.dequantize(out_c[:n // 2], out_s[:n // BLOCK], n, "e2m1", BLOCK, dst=y)
     for _ in range(3):
         mxq.fake_quant(x, "e2m3", BLOCK, mxq.FQ_VIA_ANCHOR, dst=y)
-    # the two single launches that dominate the headline step, on one decoder layer's worth of weights
-    sizes = [r * c for _, r, c in inputs.LLAMA8B_LAYER]
+    # the two single launches that dominate the headline step, on two decoder layers' worth of weights
+    sizes = [r * c for _, r, c in inputs.LLAMA8B_LAYER] * 2
+    while sum(sizes) > n:
+        sizes.pop()
     offs = np.concatenate([[0], np.cumsum(sizes)])
     pairs = [(x[int(offs[k]):int(offs[k + 1])], y[int(offs[k]):int(offs[k + 1])]) for k in range(len(sizes))]
     table = mxq.make_fq_items(pairs)
@@ -1048,6 +1068,8 @@ def main():
     ap.add_argument("--min-log2", type=int, default=16)
     ap.add_argument("--max-log2", type=int, default=31)
     ap.add_argument("--buffer-sets", type=int, default=4, help="rotating buffer sets of workload 2 (>= 2)")
+    ap.add_argument("--case-log2", type=int, default=30,
+                    help="--impl ncu-case: 2^N codes for Slice-and-Scale, 2^(N-1) elements for the other kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -213,6 +213,35 @@ int mxq_fake_quant_batched(const mxq_fq_item *items, int count, int dtype, int f
                            mxq_stream stream);
 
 /*
+ * mxq_quantize and mxq_dequantize over `count` tensors in one launch each: the anchor checkpoint of a
+ * whole model (Sec. 3.5: W_A = Q_A(W_fp) for every quantized weight, Eq. 1-3) and the reconstruction
+ * V^ = X P (Sec. 3.3, Notation) of a whole converted weight set.  `items` is a HOST array, free to
+ * reuse when the call returns; every pointer inside is a device pointer with the requirements of the
+ * single-tensor call, and the results are those of `count` single-tensor calls.  All tensors share
+ * dtype, format and block.  The item table travels in the kernel's parameter space, 512 tensors per
+ * launch (more: more launches); nothing is allocated on the device.
+ */
+typedef struct {
+    const void *src;      /* [in]  device, n elements of src_dtype */
+    size_t n;
+    void *codes;          /* [out] device, mxq_codes_bytes(n, fmt) bytes */
+    uint8_t *scales;      /* [out] device, n / block bytes */
+} mxq_q_item;
+
+int mxq_quantize_batched(const mxq_q_item *items, int count, int src_dtype, int fmt, int block,
+                         mxq_stream stream);
+
+typedef struct {
+    const void *codes;      /* [in]  device, packed codes of n elements */
+    const uint8_t *scales;  /* [in]  device, n / block bytes */
+    size_t n;
+    void *dst;              /* [out] device, n elements of dst_dtype */
+} mxq_dq_item;
+
+int mxq_dequantize_batched(const mxq_dq_item *items, int count, int fmt, int block, int dst_dtype,
+                           mxq_stream stream);
+
+/*
  * Straight-through estimator backward of mxq_fake_quant (Sec. 3.5): grad_in = grad_out.
  * grad_in == grad_out is a no-op; otherwise n elements of `dtype` are copied.
  */

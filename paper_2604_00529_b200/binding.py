@@ -34,6 +34,14 @@ class _FqItem(ctypes.Structure):
     _fields_ = [("src", ctypes.c_void_p), ("dst", ctypes.c_void_p), ("n", ctypes.c_size_t)]
 
 
+class _QItem(ctypes.Structure):
+    _fields_ = [("src", ctypes.c_void_p), ("n", ctypes.c_size_t), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p)]
+
+
+class _DqItem(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("n", ctypes.c_size_t), ("dst", ctypes.c_void_p)]
+
+
 class _Item(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("n", ctypes.c_size_t),
                 ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p)]
@@ -79,6 +87,10 @@ def load_library() -> ctypes.CDLL:
     L.mxq_fake_quant.argtypes = [vp, i, sz, i, i, i, vp, vp]
     L.mxq_fake_quant_batched.argtypes = [ctypes.POINTER(_FqItem), i, i, i, i, i, vp]
     L.mxq_fake_quant_batched.restype = i
+    L.mxq_quantize_batched.argtypes = [ctypes.POINTER(_QItem), i, i, i, i, vp]
+    L.mxq_quantize_batched.restype = i
+    L.mxq_dequantize_batched.argtypes = [ctypes.POINTER(_DqItem), i, i, i, i, vp]
+    L.mxq_dequantize_batched.restype = i
     L.mxq_tiled_scales_bytes.argtypes = [sz, sz]
     L.mxq_tiled_scales_bytes.restype = sz
     L.mxq_tile_scales.argtypes = [vp, sz, sz, vp, vp]
@@ -295,6 +307,68 @@ def fake_quant_batched(pairs, fmt: str, block: int = 32, mode: int = FQ_DIRECT, 
     table = pairs if isinstance(pairs, FqTable) else FqTable(pairs)
     _check(L.mxq_fake_quant_batched(table.array, len(table), table.dtype, FORMATS[fmt], block, mode, _stream(stream)),
            "mxq_fake_quant_batched")
+
+
+class QTable:
+    """A marshalled mxq_q_item array over (src, codes, scales) tensor triples that persist (keeps them alive)."""
+
+    def __init__(self, triples):
+        self.tensors = list(triples)
+        if not self.tensors:
+            raise ValueError("no tensors")
+        self.dtype = _dtype_id(self.tensors[0][0])
+        self.array = (_QItem * len(self.tensors))()
+        for k, (src, codes, scales) in enumerate(self.tensors):
+            if _dtype_id(src) != self.dtype:
+                raise TypeError("all tensors of a batch share one dtype")
+            self.array[k] = _QItem(_dev(src, "src"), src.numel(), _dev(codes, "codes"), _dev(scales, "scales"))
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_q_items(triples) -> QTable:
+    """Marshal (src, codes, scales) tensor triples into an mxq_q_item array."""
+    return QTable(triples)
+
+
+def quantize_batched(triples, fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_quantize_batched over (src, codes, scales) triples or a QTable made from them."""
+    L = load_library()
+    table = triples if isinstance(triples, QTable) else QTable(triples)
+    _check(L.mxq_quantize_batched(table.array, len(table), table.dtype, FORMATS[fmt], block, _stream(stream)),
+           "mxq_quantize_batched")
+
+
+class DqTable:
+    """A marshalled mxq_dq_item array over (codes, scales, n, dst) tuples that persist (keeps them alive)."""
+
+    def __init__(self, items):
+        self.tensors = list(items)
+        if not self.tensors:
+            raise ValueError("no tensors")
+        self.dtype = _dtype_id(self.tensors[0][3])
+        self.array = (_DqItem * len(self.tensors))()
+        for k, (codes, scales, n, dst) in enumerate(self.tensors):
+            if _dtype_id(dst) != self.dtype or dst.numel() != n:
+                raise TypeError("all outputs of a batch share one dtype and hold n elements")
+            self.array[k] = _DqItem(_dev(codes, "codes"), _dev(scales, "scales"), n, _dev(dst, "dst"))
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_dq_items(items) -> DqTable:
+    """Marshal (codes, scales, n, dst) tuples into an mxq_dq_item array."""
+    return DqTable(items)
+
+
+def dequantize_batched(items, fmt: str, block: int = 32, stream=None) -> None:
+    """mxq_dequantize_batched over (codes, scales, n, dst) tuples or a DqTable made from them."""
+    L = load_library()
+    table = items if isinstance(items, DqTable) else DqTable(items)
+    _check(L.mxq_dequantize_batched(table.array, len(table), FORMATS[fmt], block, table.dtype, _stream(stream)),
+           "mxq_dequantize_batched")
 
 
 def fake_quant_bwd(grad_out: torch.Tensor, grad_in: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

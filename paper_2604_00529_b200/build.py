@@ -3,7 +3,7 @@
     python -m paper_2604_00529_b200.build [--force]
 
 One object per translation unit under ``_build/`` (compiled in parallel), linked into
-``paper_2604_00529_b200/libmxq.so``.  A unit is rebuilt when it or any header is newer than
+``paper_2604_00529_b200/libmxq.so``; then ``mxq_abi_timing``, a small C-level caller of the ABI.  A unit is rebuilt when it or any header is newer than
 its object.
 """
 from __future__ import annotations
@@ -18,6 +18,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libmxq.so")
+TIMING_EXE = os.path.join(HERE, "mxq_abi_timing")      # C-level caller of the ABI (csrc/abi_timing.cu)
 UNITS = ["mxq_api", "mxq_quantize", "mxq_slice_scale", "mxq_dequantize", "mxq_fake_quant", "mxq_static_batch", "mxq_slice_scale_multi", "mxq_layout", "mxq_fake_quant_batched"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++20", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
@@ -71,6 +72,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
         tmp = LIB + ".tmp.%d" % os.getpid()
         run([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
         os.replace(tmp, LIB)
+    timing_src = os.path.join(CSRC, "abi_timing.cu")
+    if os.path.exists(timing_src) and (force or _stale(TIMING_EXE, [timing_src, LIB, os.path.join(ROOT, "include", "mxq.h")])):
+        tmp = TIMING_EXE + ".tmp.%d" % os.getpid()
+        run([_nvcc(), "-O2", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", timing_src, "-o", tmp,
+             "-L" + HERE, "-lmxq", "-Xlinker", "-rpath", "-Xlinker", "$ORIGIN"])
+        os.replace(tmp, TIMING_EXE)
     return LIB
 
 

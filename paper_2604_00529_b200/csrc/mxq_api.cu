@@ -186,6 +186,92 @@ int mxq_fake_quant_batched(const mxq_fq_item* items, int count, int dtype, int f
     return flush();
 }
 
+int mxq_quantize_batched(const mxq_q_item* items, int count, int src_dtype, int fmt, int block, mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(src_dtype)) return MXQ_ERR_FORMAT;
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+    const size_t epl = src_dtype == MXQ_F32 ? 8 : 16;       // elements per 32-byte lane unit
+    for (int i = 0; i < count; ++i) {
+        const mxq_q_item& it = items[i];
+        if (it.n % (size_t)block) return MXQ_ERR_SIZE;
+        if (it.n == 0) continue;
+        if (!it.src || !it.codes || !it.scales) return MXQ_ERR_NULL;
+        if (!aligned(it.src, 32) || !aligned(it.codes, 32) || !aligned(it.scales, 16)) return MXQ_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<QDeviceItem> chunk;
+    chunk.reserve(kQBatchItemsMax);
+    size_t tiles = 0;
+    auto flush = [&]() -> int {
+        if (chunk.empty()) return MXQ_OK;
+        const int rc = launch_quantize_batched(chunk.data(), (int)chunk.size(), tiles, src_dtype, fmt, block, s);
+        chunk.clear();
+        tiles = 0;
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const mxq_q_item& it = items[i];
+        if (it.n == 0) continue;
+        QDeviceItem d;
+        d.src = static_cast<const uint8_t*>(it.src);
+        d.codes = static_cast<uint8_t*>(it.codes);
+        d.scales = it.scales;
+        d.nunits = it.n / epl;
+        d.tile_begin = tiles;
+        tiles += q_batched_tiles(d.nunits);
+        chunk.push_back(d);
+        if ((int)chunk.size() == kQBatchItemsMax)
+            if (int rc = flush()) return rc;
+    }
+    return flush();
+}
+
+int mxq_dequantize_batched(const mxq_dq_item* items, int count, int fmt, int block, int dst_dtype, mxq_stream stream)
+{
+    if (!valid_format(fmt) || !valid_dtype(dst_dtype)) return MXQ_ERR_FORMAT;
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+    for (int i = 0; i < count; ++i) {
+        const mxq_dq_item& it = items[i];
+        if (it.n % (size_t)block || it.n % 32) return MXQ_ERR_SIZE;
+        if (it.n == 0) continue;
+        if (!it.codes || !it.scales || !it.dst) return MXQ_ERR_NULL;
+        if (!aligned(it.codes, 32) || !aligned(it.dst, 32) || !aligned(it.scales, 16)) return MXQ_ERR_ALIGN;
+    }
+    const size_t epu = dst_dtype == MXQ_F32 ? 8 : 32;        // elements per lane unit of the kernel that writes dst_dtype
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<DqDeviceItem> chunk;
+    chunk.reserve(kDqBatchItemsMax);
+    size_t tiles = 0;
+    auto flush = [&]() -> int {
+        if (chunk.empty()) return MXQ_OK;
+        const int rc = launch_dequantize_batched(chunk.data(), (int)chunk.size(), tiles, fmt, block, dst_dtype, s);
+        chunk.clear();
+        tiles = 0;
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const mxq_dq_item& it = items[i];
+        if (it.n == 0) continue;
+        DqDeviceItem d;
+        d.codes = static_cast<const uint8_t*>(it.codes);
+        d.scales = it.scales;
+        d.dst = static_cast<uint8_t*>(it.dst);
+        d.nunits = it.n / epu;
+        d.tile_begin = tiles;
+        tiles += dq_batched_tiles(d.nunits);
+        chunk.push_back(d);
+        if ((int)chunk.size() == kDqBatchItemsMax)
+            if (int rc = flush()) return rc;
+    }
+    return flush();
+}
+
 int mxq_fake_quant_bwd(const void* grad_out, int dtype, size_t n, void* grad_in, mxq_stream stream)
 {
     if (!valid_dtype(dtype)) return MXQ_ERR_FORMAT;

@@ -34,7 +34,48 @@ int run(const void* codes, const uint8_t* scales, size_t n, int block, void* dst
     }
 }
 
+// shift / scales-per-unit of the kernel that writes T (see run above)
+template <class T>
+void scale_geometry(int block, int& shift, int& per_unit)
+{
+    shift = 0;
+    per_unit = 1;
+    if constexpr (T::size == 4) {
+        while ((T::epl << shift) < block) ++shift;
+    } else {
+        if (block == 16) per_unit = 2;
+        else while ((32 << shift) < block) ++shift;
+    }
+}
+
+template <class F, class T>
+int run_batched(const DqDeviceItem* items_host, int count, size_t total_tiles, int block, cudaStream_t stream)
+{
+    DqItemBlock<kDqBatchItemsMax> blk;
+    for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
+    for (int i = count; i < kDqBatchItemsMax; ++i) blk.items[i] = DqDeviceItem{};
+    build_tile_index(blk.index, items_host, count, total_tiles);
+    int shift, per_unit;
+    scale_geometry<T>(block, shift, per_unit);
+    auto kern = dequantize_batched_kernel<F, T, kU, kThreads, kDqBatchItemsMax>;
+    return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles, shift,
+                         per_unit);
+}
+
 }  // namespace
+
+size_t dq_batched_tiles(size_t nunits) { return (nunits + 32 * kU - 1) / (32 * kU); }
+
+int launch_dequantize_batched(const DqDeviceItem* items_host, int count, size_t total_tiles, int fmt, int block, int dtype,
+                              cudaStream_t stream)
+{
+    if (count > kDqBatchItemsMax) return MXQ_ERR_SIZE;
+    MXQ_DISPATCH_FORMAT(fmt, {
+        if (dtype == MXQ_F32) return run_batched<F, F32>(items_host, count, total_tiles, block, stream);
+        return run_batched<F, BF16>(items_host, count, total_tiles, block, stream);
+    });
+    return MXQ_ERR_FORMAT;
+}
 
 int launch_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, int block, void* dst, int dtype,
                       cudaStream_t stream)

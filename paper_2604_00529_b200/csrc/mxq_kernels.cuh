@@ -316,60 +316,75 @@ __device__ __forceinline__ void quantize_unit(const uint32_t (&w)[8], float inv,
     }
 }
 
-template <class T, class F, int BLOCK, int U, int THREADS, class SCALES = uint8_t*>
-__global__ void __launch_bounds__(THREADS)
-quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes, SCALES scales)
+// One warp tile (32 U lane units) of one tensor; shared by the single-tensor and the batched kernels.
+// Every lane of the warp must call it (the block maxima meet by shuffles).
+template <class T, class F, int BLOCK, int U, class SCALES>
+__device__ __forceinline__ void quantize_tile(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes,
+                                              const SCALES& scales, size_t tile, uint8_t* stage)
 {
-    pdl_release();
     constexpr int LPB = BLOCK / T::epl;                 // lanes per block
     static_assert(LPB >= 1 && LPB <= 32, "block must cover at least one lane unit");
     constexpr int OB = T::epl * F::bits / 8;            // code bytes per lane unit
     constexpr int NW = code_words(T::epl, F::bits);
     const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
-    uint8_t* stage = nullptr;
+    const size_t u0 = tile * (32 * U) + lane;
+    uint32_t w[U][8];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit < nunits) ld256(w[u], src + unit * 32);
+        else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[u][j] = 0;
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
+        const BlockScale s = block_scale<F>(amax);
+        uint32_t out[NW];
+        quantize_unit<T, F>(w[u], s.inv, out);
+        if (s.byte == 0xFFu) {
+#pragma unroll
+            for (int j = 0; j < NW; ++j) out[j] = 0;
+        }
+        if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + lane) * OB, out);
+        if (unit < nunits) {
+            if constexpr (!StagedTile<OB>::use) store_bytes<OB>(codes + unit * OB, out);
+            if (lane % LPB == 0) put_scale(scales, unit / LPB, s.byte);
+        }
+    }
+    if constexpr (StagedTile<OB>::use) {
+        const size_t first = tile * (32 * U), left = nunits - first;
+        flush_stage<32 * U * OB>(stage, codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
+    }
+}
+
+// The staging area of the calling warp for a quantize tile (null when a lane's code piece is stored
+// directly).  Must be called by every thread of the CTA, outside divergent code.
+template <class T, class F, int U, int THREADS>
+__device__ __forceinline__ uint8_t* quantize_stage()
+{
+    constexpr int OB = T::epl * F::bits / 8;
     if constexpr (StagedTile<OB>::use) {
         __shared__ __align__(128) uint8_t stage_area[(THREADS / 32) * 32 * U * OB];
-        stage = stage_area + (threadIdx.x >> 5) * (32 * U * OB);
+        return stage_area + (threadIdx.x >> 5) * (32 * U * OB);
+    } else {
+        return nullptr;
     }
+}
 
-    prefetch_tile<U, 32>(src, warp, nunits);
+template <class T, class F, int BLOCK, int U, int THREADS, class SCALES = uint8_t*>
+__global__ void __launch_bounds__(THREADS)
+quantize_kernel(const uint8_t* __restrict__ src, size_t nunits, uint8_t* __restrict__ codes, SCALES scales)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = quantize_stage<T, F, U, THREADS>();
+    prefetch_tile<U, 32>(src, tile, nunits);
     pdl_acquire();
-    if (const size_t tile = warp; tile < ntiles) {
-        const size_t u0 = tile * (32 * U) + lane;
-        uint32_t w[U][8];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit < nunits) ld256(w[u], src + unit * 32);
-            else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) w[u][j] = 0;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            const uint32_t amax = group_max<LPB>(unit_amax_bits<T>(w[u]));
-            const BlockScale s = block_scale<F>(amax);
-            uint32_t out[NW];
-            quantize_unit<T, F>(w[u], s.inv, out);
-            if (s.byte == 0xFFu) {
-#pragma unroll
-                for (int j = 0; j < NW; ++j) out[j] = 0;
-            }
-            if constexpr (StagedTile<OB>::use) store_bytes<OB>(stage + (u * 32 + lane) * OB, out);
-            if (unit < nunits) {
-                if constexpr (!StagedTile<OB>::use) store_bytes<OB>(codes + unit * OB, out);
-                if (lane % LPB == 0) put_scale(scales, unit / LPB, s.byte);
-            }
-        }
-        if constexpr (StagedTile<OB>::use) {
-            const size_t first = tile * (32 * U), left = nunits - first;
-            flush_stage<32 * U * OB>(stage, codes + first * OB, (uint32_t)(left < 32 * U ? left : 32 * U) * OB);
-        }
-    }
+    if (tile * (32 * U) < nunits) quantize_tile<T, F, BLOCK, U>(src, nunits, codes, scales, tile, stage);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -605,6 +620,36 @@ fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count,
     pdl_acquire();
     if (tile >= total_tiles) return;                      // whole warps leave together
     fake_quant_tile<T, F, BLOCK, MODE, U>(t.src, t.nunits, t.dst, tile - t.tile_begin);
+}
+
+// Q_f (Eq. 1-3) over a whole set of tensors in one launch (the anchor checkpoint of a model, Sec. 3.5:
+// every linear weight quantized once and stored): tiles of all tensors end to end, items in the parameters.
+struct QDeviceItem {
+    const uint8_t* src;
+    uint8_t* codes;
+    uint8_t* scales;
+    size_t nunits;
+    size_t tile_begin;
+};
+
+template <int K>
+struct QItemBlock {
+    QDeviceItem items[K];
+    TileIndex index;
+};
+
+template <class T, class F, int BLOCK, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS)
+quantize_batched_kernel(const __grid_constant__ QItemBlock<K> blk, int count, size_t total_tiles)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t* stage = quantize_stage<T, F, U, THREADS>();
+    const QDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
+    if (tile < total_tiles) prefetch_tile<U, 32>(t.src, tile - t.tile_begin, t.nunits);
+    pdl_acquire();
+    if (tile >= total_tiles) return;                      // whole warps leave together
+    quantize_tile<T, F, BLOCK, U>(t.src, t.nunits, t.codes, t.scales, tile - t.tile_begin, stage);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1107,97 +1152,103 @@ slice_scale_tiled_batched_kernel(const __grid_constant__ SsTiledItemBlock<K> blk
 // is 32 bytes of OUTPUT instead and every store instruction covers 1 KB of consecutive addresses
 // (98 %).  The second shape was 1 - 2 % slower than the first for BF16 outputs.
 
+template <class F, class T, int U>
+__device__ __forceinline__ void dequantize_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                size_t nunits, int units_per_scale_shift, int scales_per_unit,
+                                                uint8_t* __restrict__ dst, size_t tile)
+{
+    constexpr int IB = 4 * F::bits, NWI = IB / 4;
+    constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
+    const int lane = threadIdx.x & 31;
+    const size_t u0 = tile * (32 * U) + lane;
+    uint32_t w[U][NWI];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
+        else {
+#pragma unroll
+            for (int j = 0; j < NWI; ++j) w[u][j] = 0;
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const size_t unit = u0 + u * 32;
+        if (unit >= nunits) continue;
+        // scales_per_unit is 1 (block >= 32: one scale shared by 2^shift units) or 2 (block 16)
+        uint32_t sbyte[2];
+        if (scales_per_unit == 1) {
+            sbyte[0] = sbyte[1] = scales[unit >> units_per_scale_shift];
+        } else {
+            sbyte[0] = scales[unit * 2];
+            sbyte[1] = scales[unit * 2 + 1];
+        }
+        uint8_t* o = dst + unit * OBYTES;
+        // four 32-byte stores for FP32 (8 elements each), two for BF16 (16 elements each)
+        constexpr int EPS = 32 / T::size;
+        static_for<32 / EPS>([&](auto k) {
+            constexpr int K = decltype(k)::value;
+            const uint32_t sbk = sbyte[(K * EPS) / 16];
+            uint32_t out[8];
+            if (sbk == 0xFFu) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+            } else if (F::id == MXQ_FP8_E4M3 && T::size == 2 &&
+                       !(has_e4m3_nan(w[u][(4 * K) % NWI]) | has_e4m3_nan(w[u][(4 * K + 1) % NWI]) |
+                         has_e4m3_nan(w[u][(4 * K + 2) % NWI]) | has_e4m3_nan(w[u][(4 * K + 3) % NWI]))) {
+                // MXFP8 anchor codes (no NaN code among these 16): the widening conversion gives the
+                // exact values, one FP32 multiply applies the scale as in the generic path below
+                const float X = scale_value(sbk);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t a, b;
+                    e4m3_word_to_f16(w[u][(4 * K + j) % NWI], a, b);
+                    float f0, f1, f2, f3;
+                    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %4; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h;\n"
+                        "  mov.b32 {l, h}, %5; cvt.f32.f16 %2, l; cvt.f32.f16 %3, h; }"
+                        : "=f"(f0), "=f"(f1), "=f"(f2), "=f"(f3) : "r"(a), "r"(b));
+                    out[2 * j] = pack_bf16x2(f0 * X, f1 * X);
+                    out[2 * j + 1] = pack_bf16x2(f2 * X, f3 * X);
+                }
+            } else {
+                const float X = scale_value(sbk);
+                static_for<EPS / 2>([&](auto i) {
+                    constexpr int I = K * EPS + 2 * decltype(i)::value;
+                    const uint32_t c0 = get_code<F::bits, I>(w[u]), c1 = get_code<F::bits, I + 1>(w[u]);
+                    float y0 = decode<F>(c0) * X;
+                    float y1 = decode<F>(c1) * X;
+                    // an E4M3 NaN code reconstructs to the canonical quiet NaN
+                    bool n0 = false, n1 = false;
+                    if constexpr (F::has_nan) {
+                        n0 = (c0 & 0x7Fu) == 0x7Fu;
+                        n1 = (c1 & 0x7Fu) == 0x7Fu;
+                    }
+                    if constexpr (T::size == 4) {
+                        out[I - K * EPS] = n0 ? 0x7FC00000u : __float_as_uint(y0);
+                        out[I - K * EPS + 1] = n1 ? 0x7FC00000u : __float_as_uint(y1);
+                    } else {
+                        uint32_t p = pack_bf16x2(y0, y1);
+                        if (n0) p = (p & 0xFFFF0000u) | 0x7FC0u;
+                        if (n1) p = (p & 0x0000FFFFu) | 0x7FC00000u;
+                        out[(I - K * EPS) / 2] = p;
+                    }
+                });
+            }
+            st256(o + K * 32, out);
+        });
+    }
+}
+
 template <class F, class T, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits,
                   int units_per_scale_shift, int scales_per_unit, uint8_t* __restrict__ dst)
 {
     pdl_release();
-    constexpr int IB = 4 * F::bits, NWI = IB / 4;
-    constexpr int OBYTES = 32 * T::size;                      // 64 or 128 bytes out per lane
-    const int lane = threadIdx.x & 31;
-    const size_t warp = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
-    const size_t ntiles = (nunits + 32 * U - 1) / (32 * U);
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     pdl_acquire();
-    if (const size_t tile = warp; tile < ntiles) {
-        const size_t u0 = tile * (32 * U) + lane;
-        uint32_t w[U][NWI];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit < nunits) load_words<NWI>(w[u], codes + unit * IB);
-            else {
-#pragma unroll
-                for (int j = 0; j < NWI; ++j) w[u][j] = 0;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t unit = u0 + u * 32;
-            if (unit >= nunits) continue;
-            // scales_per_unit is 1 (block >= 32: one scale shared by 2^shift units) or 2 (block 16)
-            uint32_t sbyte[2];
-            if (scales_per_unit == 1) {
-                sbyte[0] = sbyte[1] = scales[unit >> units_per_scale_shift];
-            } else {
-                sbyte[0] = scales[unit * 2];
-                sbyte[1] = scales[unit * 2 + 1];
-            }
-            uint8_t* o = dst + unit * OBYTES;
-            // four 32-byte stores for FP32 (8 elements each), two for BF16 (16 elements each)
-            constexpr int EPS = 32 / T::size;
-            static_for<32 / EPS>([&](auto k) {
-                constexpr int K = decltype(k)::value;
-                const uint32_t sbk = sbyte[(K * EPS) / 16];
-                uint32_t out[8];
-                if (sbk == 0xFFu) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
-                } else if (F::id == MXQ_FP8_E4M3 && T::size == 2 &&
-                           !(has_e4m3_nan(w[u][(4 * K) % NWI]) | has_e4m3_nan(w[u][(4 * K + 1) % NWI]) |
-                             has_e4m3_nan(w[u][(4 * K + 2) % NWI]) | has_e4m3_nan(w[u][(4 * K + 3) % NWI]))) {
-                    // MXFP8 anchor codes (no NaN code among these 16): the widening conversion gives the
-                    // exact values, one FP32 multiply applies the scale as in the generic path below
-                    const float X = scale_value(sbk);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint32_t a, b;
-                        e4m3_word_to_f16(w[u][(4 * K + j) % NWI], a, b);
-                        float f0, f1, f2, f3;
-                        asm("{ .reg .b16 l, h; mov.b32 {l, h}, %4; cvt.f32.f16 %0, l; cvt.f32.f16 %1, h;\n"
-                            "  mov.b32 {l, h}, %5; cvt.f32.f16 %2, l; cvt.f32.f16 %3, h; }"
-                            : "=f"(f0), "=f"(f1), "=f"(f2), "=f"(f3) : "r"(a), "r"(b));
-                        out[2 * j] = pack_bf16x2(f0 * X, f1 * X);
-                        out[2 * j + 1] = pack_bf16x2(f2 * X, f3 * X);
-                    }
-                } else {
-                    const float X = scale_value(sbk);
-                    static_for<EPS / 2>([&](auto i) {
-                        constexpr int I = K * EPS + 2 * decltype(i)::value;
-                        const uint32_t c0 = get_code<F::bits, I>(w[u]), c1 = get_code<F::bits, I + 1>(w[u]);
-                        float y0 = decode<F>(c0) * X;
-                        float y1 = decode<F>(c1) * X;
-                        // an E4M3 NaN code reconstructs to the canonical quiet NaN
-                        bool n0 = false, n1 = false;
-                        if constexpr (F::has_nan) {
-                            n0 = (c0 & 0x7Fu) == 0x7Fu;
-                            n1 = (c1 & 0x7Fu) == 0x7Fu;
-                        }
-                        if constexpr (T::size == 4) {
-                            out[I - K * EPS] = n0 ? 0x7FC00000u : __float_as_uint(y0);
-                            out[I - K * EPS + 1] = n1 ? 0x7FC00000u : __float_as_uint(y1);
-                        } else {
-                            uint32_t p = pack_bf16x2(y0, y1);
-                            if (n0) p = (p & 0xFFFF0000u) | 0x7FC0u;
-                            if (n1) p = (p & 0x0000FFFFu) | 0x7FC00000u;
-                            out[(I - K * EPS) / 2] = p;
-                        }
-                    });
-                }
-                st256(o + K * 32, out);
-            });
-        }
-    }
+    if (tile * (32 * U) < nunits)
+        dequantize_tile<F, T, U>(codes, scales, nunits, units_per_scale_shift, scales_per_unit, dst, tile);
 }
 
 
@@ -1205,18 +1256,14 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
 // of a warp covers 1 KB of consecutive addresses; the codes of a unit are 2 x bits or bits bytes,
 // read with the widest access their alignment allows.  A unit never straddles a block (blocks are
 // at least 16 elements), so it needs one scale: scales[unit >> scale_shift].
-template <class F, class T, int U, int THREADS>
-__global__ void __launch_bounds__(THREADS)
-dequantize_wide_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits, int scale_shift,
-                       uint8_t* __restrict__ dst)
+template <class F, class T, int U>
+__device__ __forceinline__ void dequantize_wide_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                     size_t nunits, int scale_shift, uint8_t* __restrict__ dst, size_t tile)
 {
-    pdl_release();
     constexpr int EPL = T::epl;                               // elements per lane unit
     constexpr int IB = EPL * F::bits / 8;                     // code bytes per lane unit
     constexpr int NWI = (IB + 3) / 4;
-    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t u0 = tile * (32 * U) + (threadIdx.x & 31);
-    pdl_acquire();
     uint32_t w[U][NWI];
     uint32_t sb[U];
 #pragma unroll
@@ -1263,6 +1310,47 @@ dequantize_wide_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
         }
         if (unit < nunits) st256(dst + unit * 32, out);
     }
+}
+
+template <class F, class T, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+dequantize_wide_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits, int scale_shift,
+                       uint8_t* __restrict__ dst)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    pdl_acquire();
+    if (tile * (32 * U) < nunits) dequantize_wide_tile<F, T, U>(codes, scales, nunits, scale_shift, dst, tile);
+}
+
+// Reconstruction of a whole set of tensors in one launch (tiles end to end, items in the parameters).
+// `shift` and `scales_per_unit` are those of the single-tensor kernel of the same output type.
+struct DqDeviceItem {
+    const uint8_t* codes;
+    const uint8_t* scales;
+    uint8_t* dst;
+    size_t nunits;
+    size_t tile_begin;
+};
+
+template <int K>
+struct DqItemBlock {
+    DqDeviceItem items[K];
+    TileIndex index;
+};
+
+template <class F, class T, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS)
+dequantize_batched_kernel(const __grid_constant__ DqItemBlock<K> blk, int count, size_t total_tiles, int shift,
+                          int scales_per_unit)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    const DqDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
+    pdl_acquire();
+    if (tile >= total_tiles) return;
+    if constexpr (T::size == 4) dequantize_wide_tile<F, T, U>(t.codes, t.scales, t.nunits, shift, t.dst, tile - t.tile_begin);
+    else dequantize_tile<F, T, U>(t.codes, t.scales, t.nunits, shift, scales_per_unit, t.dst, tile - t.tile_begin);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -46,6 +46,19 @@ int launch_fake_quant_batched(const FqDeviceItem* items_host, int count, size_t 
                               int block, int mode, cudaStream_t stream);
 size_t fq_batched_tiles(size_t nunits);
 int launch_copy(const void* src, size_t nbytes, void* dst, cudaStream_t stream);
+// Q_f and the reconstruction over up to 512 tensors in one launch; `items_host` is a HOST array whose
+// tile_begin fields are filled in (tiles counted by q_batched_tiles / dq_batched_tiles of each tensor's
+// lane units: n / elements-per-32-bytes of the source for Q_f and for FP32 outputs, n / 32 for BF16 outputs).
+struct QDeviceItem;
+struct DqDeviceItem;
+constexpr int kQBatchItemsMax = 512;
+constexpr int kDqBatchItemsMax = 512;
+int launch_quantize_batched(const QDeviceItem* items_host, int count, size_t total_tiles, int dtype, int fmt, int block,
+                            cudaStream_t stream);
+int launch_dequantize_batched(const DqDeviceItem* items_host, int count, size_t total_tiles, int fmt, int block, int dtype,
+                              cudaStream_t stream);
+size_t q_batched_tiles(size_t nunits);
+size_t dq_batched_tiles(size_t nunits);
 
 // Batched Slice-and-Scale over a device-resident item table and its coarse tile index (see
 // mxq_kernels.cuh: SsDeviceItem, TileIndex); used by the fixed-table entry point.

@@ -36,6 +36,33 @@ int by_block(int block, const void* src, size_t n, void* codes, uint8_t* scales,
     }
 }
 
+template <class T, class F, int BLOCK>
+int run_batched(const QDeviceItem* items_host, int count, size_t total_tiles, cudaStream_t stream)
+{
+    if constexpr (BLOCK < T::epl) {
+        return MXQ_ERR_BLOCK;
+    } else {
+        QItemBlock<kQBatchItemsMax> blk;
+        for (int i = 0; i < count; ++i) blk.items[i] = items_host[i];
+        for (int i = count; i < kQBatchItemsMax; ++i) blk.items[i] = QDeviceItem{};
+        build_tile_index(blk.index, items_host, count, total_tiles);
+        auto kern = quantize_batched_kernel<T, F, BLOCK, kU, kThreads, kQBatchItemsMax>;
+        return launch_kernel(kern, grid_for_tiles(total_tiles, kThreads), kThreads, stream, blk, count, total_tiles);
+    }
+}
+
+template <class T, class F>
+int batched_by_block(int block, const QDeviceItem* items_host, int count, size_t total_tiles, cudaStream_t stream)
+{
+    switch (block) {
+    case 16: return run_batched<T, F, 16>(items_host, count, total_tiles, stream);
+    case 32: return run_batched<T, F, 32>(items_host, count, total_tiles, stream);
+    case 64: return run_batched<T, F, 64>(items_host, count, total_tiles, stream);
+    case 128: return run_batched<T, F, 128>(items_host, count, total_tiles, stream);
+    default: return MXQ_ERR_BLOCK;
+    }
+}
+
 template <class T, class F>
 int run_tiled(const void* src, size_t n, void* codes, const TiledScales& tiled, cudaStream_t stream)
 {
@@ -59,6 +86,19 @@ int launch_quantize_tiled(const void* src, int dtype, size_t n, int fmt, void* c
     MXQ_DISPATCH_FORMAT(fmt, {
         if (dtype == MXQ_F32) return run_tiled<F32, F>(src, n, codes, sink, stream);
         return run_tiled<BF16, F>(src, n, codes, sink, stream);
+    });
+    return MXQ_ERR_FORMAT;
+}
+
+size_t q_batched_tiles(size_t nunits) { return (nunits + 32 * kU - 1) / (32 * kU); }
+
+int launch_quantize_batched(const QDeviceItem* items_host, int count, size_t total_tiles, int dtype, int fmt, int block,
+                            cudaStream_t stream)
+{
+    if (count > kQBatchItemsMax) return MXQ_ERR_SIZE;
+    MXQ_DISPATCH_FORMAT(fmt, {
+        if (dtype == MXQ_F32) return batched_by_block<F32, F>(block, items_host, count, total_tiles, stream);
+        return batched_by_block<BF16, F>(block, items_host, count, total_tiles, stream);
     });
     return MXQ_ERR_FORMAT;
 }

@@ -127,6 +127,27 @@ def test_argument_checks_answer_on_the_host(L):
     assert fqb(None, 3, 1, F["e2m1"], 48, 0, None) == E_BLOCK
     assert fqb(None, 3, 1, 77, 32, 0, None) == E_FORMAT
     assert fqb(None, 3, 1, F["e2m1"], 32, 5, None) == E_FORMAT
+    from paper_2604_00529_b200.binding import _DqItem, _QItem
+    qb = L.mxq_quantize_batched                      # (items, count, dtype, fmt, block, stream)
+    assert qb(None, 0, 1, F["int8"], 32, None) == OK
+    assert qb(None, 3, 1, F["int8"], 32, None) == E_NULL
+    assert qb(None, -1, 1, F["int8"], 32, None) == E_SIZE
+    assert qb(None, 3, 1, F["int8"], 48, None) == E_BLOCK
+    assert qb(None, 3, 7, F["int8"], 32, None) == E_FORMAT
+    assert qb(None, 3, 1, 99, 32, None) == E_FORMAT
+    assert qb((_QItem * 1)(_QItem(A, 48, A, A)), 1, 1, F["int8"], 32, None) == E_SIZE
+    assert qb((_QItem * 1)(_QItem(A, 64, None, A)), 1, 1, F["int8"], 32, None) == E_NULL
+    assert qb((_QItem * 1)(_QItem(A + 16, 64, A, A)), 1, 1, F["int8"], 32, None) == E_ALIGN
+    assert qb((_QItem * 1)(_QItem(None, 0, None, None)), 1, 1, F["int8"], 32, None) == OK    # empty tensor: nothing to do
+    dqb = L.mxq_dequantize_batched                   # (items, count, fmt, block, dtype, stream)
+    assert dqb(None, 0, F["int4"], 32, 1, None) == OK
+    assert dqb(None, 2, F["int4"], 32, 1, None) == E_NULL
+    assert dqb(None, -1, F["int4"], 32, 1, None) == E_SIZE
+    assert dqb(None, 2, F["int4"], 24, 1, None) == E_BLOCK
+    assert dqb(None, 2, F["int4"], 32, 3, None) == E_FORMAT
+    assert dqb((_DqItem * 1)(_DqItem(A, A, 16, A)), 1, F["int4"], 16, 1, None) == E_SIZE      # packed codes: multiples of 32
+    assert dqb((_DqItem * 1)(_DqItem(A, None, 64, A)), 1, F["int4"], 32, 1, None) == E_NULL
+    assert dqb((_DqItem * 1)(_DqItem(A, A + 8, 64, A)), 1, F["int4"], 32, 1, None) == E_ALIGN
     bw = L.mxq_fake_quant_bwd
     assert bw(A, 1, 64, A, None) == OK                                       # in place: no launch
     assert bw(A, 1, 64, None, None) == E_NULL

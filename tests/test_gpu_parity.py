@@ -370,6 +370,47 @@ def test_fake_quant_batched_matches_oracle(count, bf16):
         assert bits_equal(got, want), first_diff(got, want)
 
 
+@pytest.mark.parametrize("count", [1, 6, 512, 513, 1030])
+@pytest.mark.parametrize("fmt,bf16,block", [("int8", True, 32), ("e4m3", False, 32), ("int6", True, 64), ("e2m1", False, 16),
+                                             ("int7", True, 32), ("e3m3", True, 128)])
+def test_quantize_and_dequantize_batched_match_oracle(count, fmt, bf16, block):
+    """Whole sets of tensors of different sizes (down to one block) in one call each: Q_f into codes and
+    scales, then the reconstruction of those, both against the oracle per tensor; counts on both sides
+    of the 512-tensor launch limit; guard zones around every output."""
+    rng = np.random.default_rng(count * 131 + block)
+    per = 128 // block if block < 32 else 1                    # keep n a multiple of 32 for the packed readers
+    nblks = rng.integers(1, 24, count) * max(1, 32 // block) * per
+    if count <= 6:
+        nblks[0] = 2051 * max(1, 32 // block)                  # one tensor of many tiles and a ragged tail
+    xs, triples, items, keep = [], [], [], []
+    for k, nb in enumerate(nblks):
+        x = _mixed_f32(int(nb), 2000 + k, block)
+        if bf16:
+            x = inputs.to_bf16_bits(x)
+        n = x.size
+        c, s = Guarded(mxq.codes_bytes(n, fmt)), Guarded(n // block)
+        y = Guarded(n * (2 if k % 2 else 4), torch.bfloat16 if k % 2 else torch.float32)
+        xs.append(x)
+        triples.append((to_dev(x), c.view, s.view))
+        keep.append((c, s, y))
+    mxq.quantize_batched(triples, fmt, block)
+    # reconstruction: the even tensors to FP32 in one call, the odd ones to BF16 in another
+    for parity in (0, 1):
+        sel = [(keep[k][0].view, keep[k][1].view, xs[k].size, keep[k][2].view) for k in range(count) if k % 2 == parity]
+        if sel:
+            mxq.dequantize_batched(sel, fmt, block)
+    torch.cuda.synchronize()
+    for k, x in enumerate(xs):
+        c, s, y = keep[k]
+        for g in (c, s, y):
+            g.check()
+        wc, ws = orc.quantize(x, fmt, block)
+        assert bits_equal(to_host(s.view), ws), (k, first_diff(to_host(s.view), ws))
+        assert bits_equal(to_host(c.view), orc.pack(wc, orc.bits(fmt))), k
+        want = orc.dequantize(wc, ws, fmt, block, orc.BF16 if k % 2 else orc.F32)
+        assert bits_equal(to_host(y.view), want), (k, first_diff(to_host(y.view), want))
+
+
 # ---------------------------------------------------------------------------------------------
 # chained entry points and degenerate sizes
 # ---------------------------------------------------------------------------------------------
