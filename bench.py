@@ -514,6 +514,32 @@ def workload5(bench: Bench, device, min_log2: int, max_log2: int):
     return out
 
 
+def small_end_abi(device_index: int):
+    """The small end of the sweep through the C ABI alone: `mxq_abi_timing` (built with the library)
+    calls the entry points in a loop from C and reports, per operation and size, the host's time to
+    enqueue a call and the device's time per launch.  Returns its records, or a note when it is missing."""
+    exe = os.path.join(ROOT, "paper_2604_00529_b200", "mxq_abi_timing")
+    if not os.path.exists(exe):
+        return {"unavailable": "mxq_abi_timing is not built (python -m paper_2604_00529_b200.build)"}
+    env = dict(os.environ)
+    vis = env.get("CUDA_VISIBLE_DEVICES")
+    env["CUDA_VISIBLE_DEVICES"] = vis.split(",")[device_index] if vis else str(device_index)
+    try:
+        out = subprocess.run([exe, "16", "24", "2"], capture_output=True, text=True, timeout=300, env=env)
+    except subprocess.TimeoutExpired:
+        return {"unavailable": "mxq_abi_timing did not finish in 300 s"}
+    if out.returncode != 0:
+        return {"unavailable": "mxq_abi_timing exited with %d: %s" % (out.returncode, out.stderr.strip()[-200:])}
+    rows = {}
+    for line in out.stdout.splitlines():
+        if line.startswith("{"):
+            r = json.loads(line)
+            rows.setdefault("2^%d" % r["log2n"], {})[r["op"]] = {"host_enqueue_us": r["host_enqueue_us"],
+                                                                 "device_us": r["device_us"], "gbs": r["gbs"]}
+    return {"caller": "C program, no interpreter", "what": "per call: host time to enqueue / device time per launch, "
+            "best of 5 runs of 100 - 400 back-to-back calls over rotating cold buffers", "sizes": rows}
+
+
 # ----------------------------------------------------------------------------------------------
 # workload 3 (the headline): the 224 linear weights of an 8B Llama-shaped decoder
 # ----------------------------------------------------------------------------------------------
@@ -869,6 +895,8 @@ def run_cuda(args):
             torch.cuda.empty_cache()
         if "w5" in want:
             workloads["w5_size_sweep"] = workload5(bench, device, args.min_log2, args.max_log2)
+            torch.cuda.synchronize()
+            workloads["w5_size_sweep"]["c_abi_small_sizes"] = small_end_abi(local)
     barrier()
     sampler.stop()
     if rank != 0:

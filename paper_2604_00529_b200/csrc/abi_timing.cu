@@ -7,7 +7,7 @@
 // exceeds L2 several times over, so the figures are cold).  Small tensors are bound by whichever of
 // the two is larger.
 //
-//   mxq_abi_timing [min_log2 [max_log2]]      (defaults 16 and 24)
+//   mxq_abi_timing [min_log2 [max_log2 [step]]]      (defaults 16, 24 and 1)
 #include <chrono>
 #include <cstdio>
 #include <cstdlib>
@@ -44,8 +44,8 @@ double now_us()
 
 int main(int argc, char** argv)
 {
-    const int lo = argc > 1 ? atoi(argv[1]) : 16, hi = argc > 2 ? atoi(argv[2]) : 24;
-    if (lo < 10 || hi > 28 || lo > hi) {
+    const int lo = argc > 1 ? atoi(argv[1]) : 16, hi = argc > 2 ? atoi(argv[2]) : 24, step = argc > 3 ? atoi(argv[3]) : 1;
+    if (lo < 10 || hi > 28 || lo > hi || step < 1) {
         fprintf(stderr, "sizes 2^10 ... 2^28\n");
         return 1;
     }
@@ -56,7 +56,7 @@ int main(int argc, char** argv)
     CK(cudaEventCreate(&e1));
     const size_t l2 = 126u << 20;
 
-    for (int k = lo; k <= hi; ++k) {
+    for (int k = lo; k <= hi; k += step) {
         const size_t n = (size_t)1 << k;
         size_t copies = (4 * l2) / (2 * n) + 1;
         if (copies < 2) copies = 2;

@@ -109,14 +109,14 @@ def test_workload2_bf16_student_t_e4m3_to_fp6_fp4():
 
 # ---------------------------------------------------------------------------------------------
 # workload 3: the 224 linear weights of an 8B Llama-shaped model, converted by ONE batched launch per
-# target.  Three layers are drawn on the host (seeds 1000 layer + idx) and quantized on the GPU; the
-# other layers' anchors are device copies of those three (Slice-and-Scale is a function of the anchor
+# target.  Four layers are drawn on the host (seeds 1000 layer + idx) and quantized on the GPU; the
+# other layers' anchors are device copies of those four (Slice-and-Scale is a function of the anchor
 # codes alone, and what is checked is the anchor -> target conversion of every one of the 224 items).
 # ---------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("anchor,targets", [("int8", ("int6", "int4")), ("e4m3", ("e2m3", "e2m1"))])
 def test_workload3_whole_model_batched_conversion(anchor, targets):
-    drawn = (0, 13, 31)
+    drawn = (0, 13, 31, 7)                               # four of the 32 layers are fresh bits
     base = {}
     for li, layer in enumerate(drawn):
         for idx, (name, r, c) in enumerate(inputs.LLAMA8B_LAYER):
@@ -130,8 +130,8 @@ def test_workload3_whole_model_batched_conversion(anchor, targets):
     assert len(shapes) == 224 and sum(r * c for _, _, _, r, c in shapes) == 6979321856
     anchors = []
     for layer, idx, name, r, c in shapes:
-        src_c, src_s = base[(layer % 3, idx)]
-        if layer < 3:
+        src_c, src_s = base[(layer % len(drawn), idx)]
+        if layer < len(drawn):
             anchors.append((src_c, src_s, r * c))
         else:
             anchors.append((src_c.clone(), src_s.clone(), r * c))
@@ -189,8 +189,9 @@ def w5_base():
     return inputs.flat_bf16_normal(_W5_BASE, seed=5)
 
 
-@pytest.mark.parametrize("log2n", [16, 20, 24, 28, 31, 33])     # 33: beyond the listed sizes, element and byte
-                                                                     # offsets past 2^32
+# every size of the sweep up to 2^26 (whole tensors up to 2^20, sampled block runs above), then 2^28, the
+# 2^31 end of the sweep, and 2^33: beyond the listed sizes, element and byte offsets past 2^32
+@pytest.mark.parametrize("log2n", list(range(16, 27)) + [28, 31, 33])
 def test_workload5_size_sweep(w5_base, log2n):
     n = 1 << log2n
     base = w5_base

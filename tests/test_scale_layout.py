@@ -149,17 +149,32 @@ def test_gpu_slice_scale_tiled_batched_matches_oracle(count):
 
 @pytest.mark.gpu
 def test_gpu_tiled_entry_points_full_size_workload():
-    """BF16 8192 x 8192 (the bench's workload): fused outputs equal the two-pass outputs byte for byte
-    (the two-pass path is compared with the oracle at this size elsewhere)."""
-    x = torch.from_numpy(inputs.weight_bf16_student_t(8192, 8192, seed=1).view(np.int16)).cuda().view(torch.bfloat16)
-    x = x.view(8192, 8192)
+    """BF16 8192 x 8192 (workload 2): the fused outputs equal the two-pass outputs byte for byte, and
+    sampled bands of rows equal the oracle (Eq. 1-3, Eq. 5, then the oracle's own tiling): a band of
+    128 rows is one row of scale tiles, so its codes, plain scales and tiled bytes are contiguous slices."""
+    xb = inputs.weight_bf16_student_t(8192, 8192, seed=1)
+    x = torch.from_numpy(xb.view(np.int16)).cuda().view(torch.bfloat16).view(8192, 8192)
     codes, scales = mxq.quantize(x, "e4m3", 32)
     tc, ts = mxq.quantize_tiled(x, "e4m3", 32)
     assert torch.equal(tc, codes) and torch.equal(ts, mxq.tile_scales(scales, 8192, 256))
+    fused = {}
     for dst in ("e2m3", "e2m1"):
         lc, ls = mxq.slice_scale(codes, scales, x.numel(), "e4m3", dst, 32)
         fc, fs = mxq.slice_scale_tiled(codes, scales, 8192, 8192, "e4m3", dst, 32)
         assert torch.equal(fc, lc) and torch.equal(fs, mxq.tile_scales(ls, 8192, 256))
+        fused[dst] = (fc, fs)
+    cols, kb = 8192, 256
+    for band in (0, 17, 63):                                  # first, one in the middle, last
+        r0 = band * 128
+        xs = xb[r0 * cols:(r0 + 128) * cols]
+        wc, ws = orc.quantize(xs, "e4m3")
+        assert np.array_equal(tc[r0 * cols:(r0 + 128) * cols].cpu().numpy(), orc.pack(wc, 8)), band
+        assert np.array_equal(ts[band * 128 * kb:(band + 1) * 128 * kb].cpu().numpy(), orc.tile_scales(ws, 128, kb)), band
+        for dst, (fc, fs) in fused.items():
+            b = orc.bits(dst)
+            lc, ls = orc.slice_scale(wc, ws, "e4m3", dst)
+            assert np.array_equal(fc[r0 * cols * b // 8:(r0 + 128) * cols * b // 8].cpu().numpy(), orc.pack(lc, b)), (band, dst)
+            assert np.array_equal(fs[band * 128 * kb:(band + 1) * 128 * kb].cpu().numpy(), orc.tile_scales(ls, 128, kb)), (band, dst)
 
 
 def _mixed_matrix(rows, cols, seed):
