@@ -88,6 +88,30 @@ typedef enum {
 /* Human-readable name of a status code (static storage, never null). */
 const char *mxq_status_string(int status);
 
+/*
+ * Debug builds of the library (compiled with -DMXQ_DEBUG; `python -m paper_2604_00529_b200.build --debug`
+ * makes libmxq_debug.so) check every global-memory access of the kernels against the byte ranges of
+ * the buffers the entry point was given -- computed from n, the format's width and the block size in
+ * this layer, independently of the kernels' index arithmetic.  An access outside them is counted,
+ * its address kept, and the access skipped: nothing traps.  (The paper has no counterpart; this is
+ * the library's own sanitizer.)  Debug builds serve one stream at a time and are several times slower.
+ *   mxq_debug_report      waits for the device, fills `out`, optionally clears the counters.
+ *                         out->enabled is 0 in a release build (everything else stays 0).
+ *   mxq_debug_trim_ranges test hook: from now on this thread registers every range `bytes` short, so
+ *                         that the checker can be seen to catch the kernels' (legitimate) last accesses
+ *                         without any access leaving its real buffer.  Returns 1 in a debug build, 0 otherwise.
+ */
+typedef struct {
+    int enabled;                      /* 1: the library was built with -DMXQ_DEBUG */
+    unsigned int checked_launches;    /* launches that ran with ranges registered */
+    unsigned int violations;          /* accesses outside every registered range (each skipped) */
+    unsigned long long first_address; /* address and size of the first one seen */
+    unsigned int first_bytes;
+} mxq_debug_info;
+
+int mxq_debug_report(mxq_debug_info *out, int reset);
+int mxq_debug_trim_ranges(size_t bytes);
+
 /* Bits per element code of `fmt`, or 0 for an unknown format. */
 int mxq_format_bits(int fmt);
 

@@ -1,6 +1,6 @@
 """Builds libmxq.so (the CUDA C-ABI library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2604_00529_b200.build [--force]
+    python -m paper_2604_00529_b200.build [--force] [--debug]
 
 One object per translation unit under ``_build/`` (compiled in parallel), linked into
 ``paper_2604_00529_b200/libmxq.so``; then ``mxq_abi_timing``, a small C-level caller of the ABI.  A unit is rebuilt when it or any header is newer than
@@ -44,7 +44,18 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+DEBUG_LIB = os.path.join(HERE, "libmxq_debug.so")      # the same sources with -DMXQ_DEBUG (bounds-checked accesses)
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds libmxq.so (and mxq_abi_timing); with debug=True builds libmxq_debug.so instead."""
+    if debug:
+        return _build_library(os.path.join(ROOT, "_build_debug"), DEBUG_LIB, ["-DMXQ_DEBUG"], force, verbose, timing=False)
+    return _build_library(OBJ_DIR, LIB, [], force, verbose, timing=True)
+
+
+def _build_library(obj_dir: str, lib: str, extra, force: bool, verbose: bool, timing: bool) -> str:
+    OBJ_DIR, LIB = obj_dir, lib
     os.makedirs(OBJ_DIR, exist_ok=True)
     headers = _headers()
     units = [u for u in UNITS if os.path.exists(os.path.join(CSRC, u + ".cu"))]
@@ -53,7 +64,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         src = os.path.join(CSRC, u + ".cu")
         obj = os.path.join(OBJ_DIR, u + ".o")
         if force or _stale(obj, [src] + headers):
-            cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+            cmd = [_nvcc()] + NVCC_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
             jobs.append(cmd)
 
     def run(cmd):
@@ -73,7 +84,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         run([_nvcc(), "-shared", "-o", tmp] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
         os.replace(tmp, LIB)
     timing_src = os.path.join(CSRC, "abi_timing.cu")
-    if os.path.exists(timing_src) and (force or _stale(TIMING_EXE, [timing_src, LIB, os.path.join(ROOT, "include", "mxq.h")])):
+    if timing and os.path.exists(timing_src) and (force or _stale(TIMING_EXE, [timing_src, LIB, os.path.join(ROOT, "include", "mxq.h")])):
         tmp = TIMING_EXE + ".tmp.%d" % os.getpid()
         run([_nvcc(), "-O2", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", timing_src, "-o", tmp,
              "-L" + HERE, "-lmxq", "-Xlinker", "-rpath", "-Xlinker", "$ORIGIN"])
@@ -82,4 +93,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -5,7 +5,18 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "mxq_debug.cuh"
+
 namespace mxq {
+
+// In debug builds (-DMXQ_DEBUG) every access below is first tested against the byte ranges the entry
+// point registered (mxq_debug.cuh); one that falls outside is counted and skipped.
+#ifdef MXQ_DEBUG
+#define MXQ_CHECKED(p, bytes, on_fail) \
+    if (!::mxq::debug_ok((p), (bytes))) { on_fail; }
+#else
+#define MXQ_CHECKED(p, bytes, on_fail)
+#endif
 
 // ---- programmatic dependent launch ----------------------------------------------------------
 // Every kernel of the library is launched with programmatic stream serialization allowed: its
@@ -41,6 +52,7 @@ __device__ __forceinline__ void prefetch_tile(const uint8_t* base, size_t tile, 
 
 __device__ __forceinline__ void ld256(uint32_t (&w)[8], const void* p)
 {
+    MXQ_CHECKED(p, 32, { for (int j = 0; j < 8; ++j) w[j] = 0; return; })
     asm volatile("ld.global.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
                  : "l"(p));
@@ -48,9 +60,24 @@ __device__ __forceinline__ void ld256(uint32_t (&w)[8], const void* p)
 
 __device__ __forceinline__ void st256(void* p, const uint32_t (&w)[8])
 {
+    MXQ_CHECKED(p, 32, return)
     asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                  :: "l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                  : "memory");
+}
+
+// ---- single bytes (the scale streams) -------------------------------------------------------
+
+__device__ __forceinline__ uint32_t ld_u8(const uint8_t* p)
+{
+    MXQ_CHECKED(p, 1, return 0)
+    return *p;
+}
+
+__device__ __forceinline__ void st_u8(uint8_t* p, uint32_t v)
+{
+    MXQ_CHECKED(p, 1, return)
+    *p = (uint8_t)v;
 }
 
 // ---- compile-time sized pieces --------------------------------------------------------------
@@ -70,6 +97,9 @@ __device__ __forceinline__ void load_words(uint32_t (&w)[NW], const void* p)
 {
     constexpr int A = piece_align(NW * 4);
     const char* c = static_cast<const char*>(p);
+    if constexpr (A != 32) {                                  // (32-byte pieces are checked by ld256)
+        MXQ_CHECKED(p, NW * 4, { for (int i = 0; i < NW; ++i) w[i] = 0; return; })
+    }
     if constexpr (A == 32) {
 #pragma unroll
         for (int i = 0; i < NW; i += 8) {
@@ -110,6 +140,7 @@ __device__ __forceinline__ void load_bytes(uint32_t (&w)[NW], const void* p)
         const char* c = static_cast<const char*>(p);
 #pragma unroll
         for (int i = 0; i < NW; ++i) w[i] = 0;
+        MXQ_CHECKED(p, NB, return)
         if constexpr (A == 2) {
 #pragma unroll
             for (int i = 0; i < NB / 2; ++i)
@@ -128,6 +159,9 @@ __device__ __forceinline__ void store_bytes(void* p, const uint32_t (&w)[NW])
     static_assert(NW * 4 >= NB, "not enough words");
     constexpr int A = piece_align(NB);
     char* c = static_cast<char*>(p);
+    if constexpr (A != 32) {                                  // (32-byte pieces are checked by st256)
+        MXQ_CHECKED(p, NB, return)
+    }
     if constexpr (A == 32) {
 #pragma unroll
         for (int i = 0; i < NB / 4; i += 8) {
@@ -191,7 +225,9 @@ __device__ __forceinline__ void flush_stage(const uint8_t* stage, uint8_t* gdst,
         // waits until the engine has read the area (it may be rewritten or released afterwards)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) {
+        bool ok = true;
+        MXQ_CHECKED(gdst, TILE_BYTES, ok = false)
+        if (lane == 0 && ok) {
             const uint32_t saddr = (uint32_t)__cvta_generic_to_shared(stage);
             asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                          :: "l"(gdst), "r"(saddr), "r"(TILE_BYTES) : "memory");
@@ -202,10 +238,12 @@ __device__ __forceinline__ void flush_stage(const uint8_t* stage, uint8_t* gdst,
         return;
     }
     __syncwarp();
-    for (uint32_t i = lane * 16; i + 16 <= nbytes; i += 512)
+    for (uint32_t i = lane * 16; i + 16 <= nbytes; i += 512) {
+        MXQ_CHECKED(gdst + i, 16, continue)
         *reinterpret_cast<uint4*>(gdst + i) = *reinterpret_cast<const uint4*>(stage + i);
+    }
     const uint32_t done = nbytes & ~15u;                        // a ragged tensor end: up to 15 bytes
-    if (done + lane < nbytes) gdst[done + lane] = stage[done + lane];
+    if (done + lane < nbytes) st_u8(gdst + done + lane, stage[done + lane]);
     __syncwarp();
 }
 

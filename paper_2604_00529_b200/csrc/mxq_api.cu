@@ -48,6 +48,46 @@ const char* mxq_status_string(int status)
     }
 }
 
+int mxq_debug_report(mxq_debug_info* out, int reset)
+{
+    if (!out) return MXQ_ERR_NULL;
+    *out = mxq_debug_info{};
+#ifdef MXQ_DEBUG
+    out->enabled = 1;
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+    out->checked_launches = debug_checked_launches().load();
+    for (const DebugUnit& u : debug_units()) {
+        unsigned int v = 0, bytes = 0;
+        unsigned long long first = 0;
+        if (u.read(&v, &first, &bytes) != 0) return MXQ_ERR_CUDA;
+        if (v && !out->violations) {
+            out->first_address = first;
+            out->first_bytes = bytes;
+        }
+        out->violations += v;
+        if (reset && u.reset() != 0) return MXQ_ERR_CUDA;
+    }
+    if (reset) debug_checked_launches().store(0);
+#else
+    (void)reset;
+#endif
+    return MXQ_OK;
+}
+
+int mxq_debug_trim_ranges(size_t bytes)
+{
+#ifdef MXQ_DEBUG
+    debug_pending().trim = bytes;
+    return 1;
+#else
+    (void)bytes;
+    return 0;
+#endif
+}
+
 int mxq_format_bits(int fmt) { return valid_format(fmt) ? fmt_info(fmt).bits : 0; }
 
 size_t mxq_codes_bytes(size_t n, int fmt) { return valid_format(fmt) ? n * (size_t)fmt_info(fmt).bits / 8 : 0; }
@@ -64,6 +104,10 @@ int mxq_quantize(const void* src, int src_dtype, size_t n, int fmt, int block, v
     if (n == 0) return MXQ_OK;
     if (!src || !codes || !scales) return MXQ_ERR_NULL;
     if (!aligned(src, 32) || !aligned(codes, 32) || !aligned(scales, 16)) return MXQ_ERR_ALIGN;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(src, n * (src_dtype == MXQ_F32 ? 4u : 2u));
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(scales, n / (size_t)block);
     return launch_quantize(src, src_dtype, n, fmt, block, codes, scales, static_cast<cudaStream_t>(stream));
 }
 
@@ -78,6 +122,11 @@ int mxq_slice_scale(const void* codes, const uint8_t* scales, size_t n, int bloc
     if (!codes || !scales || !out_codes || !out_scales) return MXQ_ERR_NULL;
     if (!aligned(codes, 32) || !aligned(out_codes, 32) || !aligned(scales, 16) || !aligned(out_scales, 16))
         return MXQ_ERR_ALIGN;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(src_fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(scales, n / (size_t)block);
+    MXQ_DEBUG_EXPECT(out_codes, n * (size_t)fmt_info(dst_fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(out_scales, n / (size_t)block);
     return launch_slice_scale(codes, scales, n, block, src_fmt, dst_fmt, out_codes, out_scales,
                               static_cast<cudaStream_t>(stream));
 }
@@ -101,6 +150,13 @@ int mxq_slice_scale_multi(const void* codes, const uint8_t* scales, size_t n, in
     for (int t = 0; t < ntargets; ++t) {
         if (!out_codes[t] || !out_scales[t]) return MXQ_ERR_NULL;
         if (!aligned(out_codes[t], 32) || !aligned(out_scales[t], 16)) return MXQ_ERR_ALIGN;
+    }
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(src_fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(scales, n / (size_t)block);
+    for (int k = 0; k < ntargets; ++k) {
+        MXQ_DEBUG_EXPECT(out_codes[k], n * (size_t)fmt_info(dst_fmts[k]).bits / 8);
+        MXQ_DEBUG_EXPECT(out_scales[k], n / (size_t)block);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int t = 0;
@@ -127,6 +183,10 @@ int mxq_dequantize(const void* codes, const uint8_t* scales, size_t n, int fmt, 
     if (n == 0) return MXQ_OK;
     if (!codes || !scales || !dst) return MXQ_ERR_NULL;
     if (!aligned(codes, 32) || !aligned(dst, 32) || !aligned(scales, 16)) return MXQ_ERR_ALIGN;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(scales, n / (size_t)block);
+    MXQ_DEBUG_EXPECT(dst, n * (dst_dtype == MXQ_F32 ? 4u : 2u));
     return launch_dequantize(codes, scales, n, fmt, block, dst, dst_dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -138,6 +198,9 @@ int mxq_fake_quant(const void* src, int dtype, size_t n, int fmt, int block, int
     if (n == 0) return MXQ_OK;
     if (!src || !dst) return MXQ_ERR_NULL;
     if (!aligned(src, 32) || !aligned(dst, 32)) return MXQ_ERR_ALIGN;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(src, n * (dtype == MXQ_F32 ? 4u : 2u));
+    MXQ_DEBUG_EXPECT(dst, n * (dtype == MXQ_F32 ? 4u : 2u));
     return launch_fake_quant(src, dtype, n, fmt, block, mode, dst, static_cast<cudaStream_t>(stream));
 }
 
@@ -157,6 +220,11 @@ int mxq_fake_quant_batched(const mxq_fq_item* items, int count, int dtype, int f
         if (it.n == 0) continue;
         if (!it.src || !it.dst) return MXQ_ERR_NULL;
         if (!aligned(it.src, 32) || !aligned(it.dst, 32)) return MXQ_ERR_ALIGN;
+    }
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].src, items[i].n * (dtype == MXQ_F32 ? 4u : 2u));
+        MXQ_DEBUG_EXPECT(items[i].dst, items[i].n * (dtype == MXQ_F32 ? 4u : 2u));
     }
     // launches of at most kFqBatchItemsMax tensors each: the item table rides in the kernel parameters
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -201,6 +269,12 @@ int mxq_quantize_batched(const mxq_q_item* items, int count, int src_dtype, int 
         if (!it.src || !it.codes || !it.scales) return MXQ_ERR_NULL;
         if (!aligned(it.src, 32) || !aligned(it.codes, 32) || !aligned(it.scales, 16)) return MXQ_ERR_ALIGN;
     }
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].src, items[i].n * (src_dtype == MXQ_F32 ? 4u : 2u));
+        MXQ_DEBUG_EXPECT(items[i].codes, items[i].n * (size_t)fmt_info(fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, items[i].n / (size_t)block);
+    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<QDeviceItem> chunk;
     chunk.reserve(kQBatchItemsMax);
@@ -243,6 +317,12 @@ int mxq_dequantize_batched(const mxq_dq_item* items, int count, int fmt, int blo
         if (!it.codes || !it.scales || !it.dst) return MXQ_ERR_NULL;
         if (!aligned(it.codes, 32) || !aligned(it.dst, 32) || !aligned(it.scales, 16)) return MXQ_ERR_ALIGN;
     }
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].codes, items[i].n * (size_t)fmt_info(fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, items[i].n / (size_t)block);
+        MXQ_DEBUG_EXPECT(items[i].dst, items[i].n * (dst_dtype == MXQ_F32 ? 4u : 2u));
+    }
     const size_t epu = dst_dtype == MXQ_F32 ? 8 : 32;        // elements per lane unit of the kernel that writes dst_dtype
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<DqDeviceItem> chunk;
@@ -279,6 +359,9 @@ int mxq_fake_quant_bwd(const void* grad_out, int dtype, size_t n, void* grad_in,
     if (!grad_out || !grad_in) return MXQ_ERR_NULL;
     if (!aligned(grad_out, 32) || !aligned(grad_in, 32)) return MXQ_ERR_ALIGN;
     if (grad_out == grad_in) return MXQ_OK;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(grad_out, n * (dtype == MXQ_F32 ? 4u : 2u));
+    MXQ_DEBUG_EXPECT(grad_in, n * (dtype == MXQ_F32 ? 4u : 2u));
     return launch_copy(grad_out, n * (dtype == MXQ_F32 ? 4u : 2u), grad_in, static_cast<cudaStream_t>(stream));
 }
 
@@ -316,6 +399,13 @@ int mxq_slice_scale_batched(const mxq_ss_item* items, int count, int block, int 
         host.push_back(d);
     }
     if (host.empty()) return MXQ_OK;
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].codes, items[i].n * (size_t)fmt_info(src_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, items[i].n / (size_t)block);
+        MXQ_DEBUG_EXPECT(items[i].out_codes, items[i].n * (size_t)fmt_info(dst_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].out_scales, items[i].n / (size_t)block);
+    }
 
     // the item table rides in the kernel's parameter space, kSsParamItemsMax tensors per launch: nothing
     // to allocate or copy, no state shared between calls; larger sets take several launches (each

@@ -48,7 +48,7 @@ __device__ __forceinline__ void static_for(Fn&& fn)
 
 __device__ __forceinline__ void put_scale(uint8_t* scales, size_t blk, uint32_t byte)
 {
-    scales[blk] = (uint8_t)byte;
+    st_u8(scales + blk, byte);
 }
 
 // Division of a 32-bit block index by the row length in blocks, by multiply and shift (the
@@ -87,7 +87,7 @@ __host__ __device__ __forceinline__ size_t tiled_scale_offset(const TiledScales&
 
 __device__ __forceinline__ void put_scale(const TiledScales& t, size_t blk, uint32_t byte)
 {
-    t.base[tiled_scale_offset(t, blk)] = (uint8_t)byte;
+    st_u8(t.base + tiled_scale_offset(t, blk), byte);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -900,7 +900,7 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
 #pragma unroll
             for (int j = 0; j < NWI; ++j) w[u][j] = 0;
         }
-        sb[u] = unit < nscales ? scales[unit] : 0;
+        sb[u] = unit < nscales ? ld_u8(scales + unit) : 0;
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -919,7 +919,7 @@ __device__ __forceinline__ void slice_scale_tile(const uint8_t* __restrict__ cod
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const size_t i = nunits + u0 + u * 32;
-            if (i < nscales) put_scale(out_scales, i, ss_scale_byte(scales[i], de));
+            if (i < nscales) put_scale(out_scales, i, ss_scale_byte(ld_u8(scales + i), de));
         }
     }
 }
@@ -1003,14 +1003,14 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
 #pragma unroll
             for (int j = 0; j < NWI; ++j) w[u][j] = 0;
         }
-        sb[u] = unit < nscales ? scales[unit] : 0;
+        sb[u] = unit < nscales ? ld_u8(scales + unit) : 0;
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const size_t unit = u0 + u * 32;
         if (unit < nscales) {
-            out_scales1[unit] = ss_scale_byte(sb[u], de1);
-            out_scales2[unit] = ss_scale_byte(sb[u], de2);
+            st_u8(out_scales1 + unit, ss_scale_byte(sb[u], de1));
+            st_u8(out_scales2 + unit, ss_scale_byte(sb[u], de2));
         }
         uint32_t o1[OB1 / 4], o2[OB2 / 4];
         if constexpr (ss_e4m3_has_fast_path<FH, FL1>() && ss_e4m3_has_fast_path<FH, FL2>()) {
@@ -1043,9 +1043,9 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
         for (int u = 0; u < U; ++u) {
             const size_t i = nunits + u0 + u * 32;
             if (i < nscales) {
-                const uint32_t b = scales[i];
-                out_scales1[i] = ss_scale_byte(b, de1);
-                out_scales2[i] = ss_scale_byte(b, de2);
+                const uint32_t b = ld_u8(scales + i);
+                st_u8(out_scales1 + i, ss_scale_byte(b, de1));
+                st_u8(out_scales2 + i, ss_scale_byte(b, de2));
             }
         }
     }
@@ -1178,10 +1178,10 @@ __device__ __forceinline__ void dequantize_tile(const uint8_t* __restrict__ code
         // scales_per_unit is 1 (block >= 32: one scale shared by 2^shift units) or 2 (block 16)
         uint32_t sbyte[2];
         if (scales_per_unit == 1) {
-            sbyte[0] = sbyte[1] = scales[unit >> units_per_scale_shift];
+            sbyte[0] = sbyte[1] = ld_u8(scales + (unit >> units_per_scale_shift));
         } else {
-            sbyte[0] = scales[unit * 2];
-            sbyte[1] = scales[unit * 2 + 1];
+            sbyte[0] = ld_u8(scales + unit * 2);
+            sbyte[1] = ld_u8(scales + unit * 2 + 1);
         }
         uint8_t* o = dst + unit * OBYTES;
         // four 32-byte stores for FP32 (8 elements each), two for BF16 (16 elements each)
@@ -1271,7 +1271,7 @@ __device__ __forceinline__ void dequantize_wide_tile(const uint8_t* __restrict__
         const size_t unit = u0 + u * 32;
         if (unit < nunits) {
             load_bytes<IB>(w[u], codes + unit * IB);
-            sb[u] = scales[unit >> scale_shift];
+            sb[u] = ld_u8(scales + (unit >> scale_shift));
         } else {
 #pragma unroll
             for (int j = 0; j < NWI; ++j) w[u][j] = 0;
@@ -1380,7 +1380,7 @@ copy_kernel(const uint8_t* __restrict__ src, size_t nbytes, uint8_t* __restrict_
     }
     // ragged tail (n * size need not be a multiple of 32 bytes)
     const size_t tid = (size_t)blockIdx.x * THREADS + threadIdx.x;
-    for (size_t i = nunits * 32 + tid; i < nbytes; i += (size_t)gridDim.x * THREADS) dst[i] = src[i];
+    for (size_t i = nunits * 32 + tid; i < nbytes; i += (size_t)gridDim.x * THREADS) st_u8(dst + i, ld_u8(src + i));
 }
 
 }  // namespace mxq

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/mxq.h"
+#include "mxq_debug.cuh"
 
 namespace mxq {
 
@@ -106,6 +107,12 @@ template <class... KArgs, class... Args>
 inline int launch_kernel(void (*kern)(KArgs...), int grid, int threads, cudaStream_t stream, Args... args)
 {
     if (grid <= 0) return MXQ_ERR_SIZE;
+#ifdef MXQ_DEBUG
+    if (debug_upload(stream) != 0) {                      // the byte ranges this launch may touch
+        (void)cudaGetLastError();
+        return MXQ_ERR_CUDA;
+    }
+#endif
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)threads);

@@ -38,15 +38,18 @@ tile_scales_kernel(const uint8_t* __restrict__ scales, size_t rows, size_t kbloc
         if (row < rows) {
             const uint8_t* p = scales + row * kblocks + ct * 4;
             if constexpr (VEC) {
-                v = *reinterpret_cast<const uint32_t*>(p);         // kblocks % 4 == 0: in range and aligned
+                bool ok = true;
+                MXQ_CHECKED(p, 4, ok = false)
+                if (ok) v = *reinterpret_cast<const uint32_t*>(p); // kblocks % 4 == 0: in range and aligned
             } else {
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    if (ct * 4 + c < kblocks) v |= (uint32_t)p[c] << (8 * c);
+                    if (ct * 4 + c < kblocks) v |= ld_u8(p + c) << (8 * c);
             }
         }
         w[g] = v;
     }
+    MXQ_CHECKED(out + tile * 512 + (size_t)lane * 16, 16, return)
     *reinterpret_cast<uint4*>(out + tile * 512 + (size_t)lane * 16) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -98,6 +101,9 @@ int mxq_tile_scales(const uint8_t* scales, size_t rows, size_t kblocks, uint8_t*
     const size_t col_tiles = (kblocks + 3) / 4, ntiles = ((rows + 127) / 128) * col_tiles;
     const int grid = grid_for_tiles(ntiles, kThreads);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(scales, rows * kblocks);
+    MXQ_DEBUG_EXPECT(tiled, tiled_bytes(rows, kblocks));
     if (kblocks % 4 == 0)
         return launch_kernel(tile_scales_kernel<true>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
     return launch_kernel(tile_scales_kernel<false>, grid, kThreads, s, scales, rows, kblocks, col_tiles, ntiles, tiled);
@@ -115,6 +121,10 @@ int mxq_quantize_tiled(const void* src, int src_dtype, size_t rows, size_t cols,
     if (!aligned(src, 32) || !aligned(codes, 32) || !aligned(tiled_scales, 16)) return MXQ_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (int rc = clear_partial_tiles(tiled_scales, rows, kblocks, s)) return rc;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(src, n * (src_dtype == MXQ_F32 ? 4u : 2u));
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(tiled_scales, tiled_bytes(rows, kblocks));
     return launch_quantize_tiled(src, src_dtype, n, fmt, codes, tiled_scales, kblocks, s);
 }
 
@@ -132,6 +142,11 @@ int mxq_slice_scale_tiled(const void* codes, const uint8_t* scales, size_t rows,
         return MXQ_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (int rc = clear_partial_tiles(out_tiled_scales, rows, kblocks, s)) return rc;
+    MXQ_DEBUG_SCOPE();
+    MXQ_DEBUG_EXPECT(codes, n * (size_t)fmt_info(src_fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(scales, n / 32);
+    MXQ_DEBUG_EXPECT(out_codes, n * (size_t)fmt_info(dst_fmt).bits / 8);
+    MXQ_DEBUG_EXPECT(out_tiled_scales, tiled_bytes(rows, kblocks));
     return launch_slice_scale_tiled(codes, scales, n, src_fmt, dst_fmt, out_codes, out_tiled_scales, kblocks, s);
 }
 
@@ -155,6 +170,14 @@ int mxq_slice_scale_tiled_batched(const mxq_ss_tiled_item* items, int count, int
         if (!aligned(it.codes, 32) || !aligned(it.out_codes, 32) || !aligned(it.scales, 16) ||
             !aligned(it.out_tiled_scales, 16))
             return MXQ_ERR_ALIGN;
+    }
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        const size_t n = items[i].rows * items[i].cols;
+        MXQ_DEBUG_EXPECT(items[i].codes, n * (size_t)fmt_info(src_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, n / 32);
+        MXQ_DEBUG_EXPECT(items[i].out_codes, n * (size_t)fmt_info(dst_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].out_tiled_scales, tiled_bytes(items[i].rows, items[i].cols / 32));
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<SsTiledDeviceItem> chunk;

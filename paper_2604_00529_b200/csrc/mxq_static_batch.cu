@@ -95,6 +95,13 @@ extern "C" int mxq_slice_scale_batched_static(const mxq_ss_item* items, int coun
         tiles += ss_batched_tiles(d.nunits);
     }
     if (used == 0) return MXQ_OK;
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].codes, items[i].n * (size_t)fmt_info(src_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, items[i].n / (size_t)block);
+        MXQ_DEBUG_EXPECT(items[i].out_codes, items[i].n * (size_t)fmt_info(dst_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].out_scales, items[i].n / (size_t)block);
+    }
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // The table copy below reads `staged`, which is gone when this function returns.  A stream that is
