@@ -649,6 +649,15 @@ def whole_model_conversions(bench: Bench, wm: WholeModel):
         out["%s_to_%s" % (a, t)] = {"batched_one_launch": bench.record(tb, nbytes, wm.total),
                                     "per_tensor_launches": bench.record(tp, nbytes, wm.total, launches_per_call=len(wm.sizes))}
         bench.launches += (REGIONS + 1) * (1 + len(wm.sizes))
+    # both lower formats of a family from ONE read of the anchor, over the whole model in one launch
+    for a, t1, t2 in (("int8", "int6", "int4"), ("e4m3", "e2m3", "e2m1")):
+        table = mxq.make_pair_items([(c, s, n, oc1, os1, oc2, os2) for (c, s, n, oc1, os1), (_, _, _, oc2, os2)
+                                     in zip(wm.ss_items[(a, t1)].tensors, wm.ss_items[(a, t2)].tensors)])
+        nbytes = (1 + SCALE_B + BITS[t1] / 8 + SCALE_B + BITS[t2] / 8 + SCALE_B) * wm.total
+        tb = bench.regions(lambda j: mxq.slice_scale_pair_batched(table, a, t1, t2, BLOCK), 1, reps=1, warm=1)
+        out["%s_to_%s_and_%s_one_read" % (a, t1, t2)] = {"batched_one_launch": bench.record(tb, nbytes, wm.total)}
+        bench.launches += REGIONS + 1
+        del table
     for f in ("int8", "e4m3"):
         nbytes = b_quantize(2, f) * wm.total
         tb = bench.regions(lambda j: mxq.quantize_batched(wm.q_tables[f], f, BLOCK), 1, reps=1, warm=1)

@@ -101,7 +101,7 @@ const char *mxq_status_string(int status);
  *                         that the checker can be seen to catch the kernels' (legitimate) last accesses
  *                         without any access leaving its real buffer.  Returns 1 in a debug build, 0 otherwise.
  */
-typedef struct {
+typedef struct mxq_debug_info {
     int enabled;                      /* 1: the library was built with -DMXQ_DEBUG */
     unsigned int checked_launches;    /* launches that ran with ranges registered */
     unsigned int violations;          /* accesses outside every registered range (each skipped) */
@@ -227,7 +227,7 @@ int mxq_fake_quant(const void *src, int dtype, size_t n, int fmt, int block, int
  * travels in the kernel's parameter space, 512 tensors per launch; more are split over several
  * launches.  Nothing is allocated on the device.
  */
-typedef struct {
+typedef struct mxq_fq_item {
     const void *src;
     void *dst;
     size_t n;
@@ -245,7 +245,7 @@ int mxq_fake_quant_batched(const mxq_fq_item *items, int count, int dtype, int f
  * dtype, format and block.  The item table travels in the kernel's parameter space, 512 tensors per
  * launch (more: more launches); nothing is allocated on the device.
  */
-typedef struct {
+typedef struct mxq_q_item {
     const void *src;      /* [in]  device, n elements of src_dtype */
     size_t n;
     void *codes;          /* [out] device, mxq_codes_bytes(n, fmt) bytes */
@@ -255,7 +255,7 @@ typedef struct {
 int mxq_quantize_batched(const mxq_q_item *items, int count, int src_dtype, int fmt, int block,
                          mxq_stream stream);
 
-typedef struct {
+typedef struct mxq_dq_item {
     const void *codes;      /* [in]  device, packed codes of n elements */
     const uint8_t *scales;  /* [in]  device, n / block bytes */
     size_t n;
@@ -280,7 +280,7 @@ int mxq_fake_quant_bwd(const void *grad_out, int dtype, size_t n, void *grad_in,
  * space, 512 non-empty tensors per launch (more tensors: more launches); nothing is
  * allocated or copied and no state is shared between calls.
  */
-typedef struct {
+typedef struct mxq_ss_item {
     const void *codes;
     const uint8_t *scales;
     size_t n;
@@ -292,6 +292,29 @@ int mxq_slice_scale_batched(const mxq_ss_item *items, int count, int block,
                             int src_fmt, int dst_fmt, mxq_stream stream);
 
 /*
+ * Whole-model conversion into TWO lower formats from one read of every anchor (Sec. 3.5, Inference: one
+ * stored anchor checkpoint, several precisions served at once; Eq. 4-5 applied twice per element): the
+ * results of mxq_slice_scale_batched to dst_fmt1 and to dst_fmt2.  For the fused pairs of
+ * mxq_slice_scale_multi one launch covers 256 tensors and reads the anchors once (2.34 instead of
+ * 3.375 bytes per element for 6-bit + 4-bit targets); any other legal pair of targets runs as two
+ * single-target batched passes.  `items` is a HOST array; requirements per pointer as in mxq_slice_scale;
+ * block must be 32, 64 or 128; outputs must not overlap the inputs or one another.  Nothing is allocated
+ * on the device.
+ */
+typedef struct mxq_ss_pair_item {
+    const void *codes;
+    const uint8_t *scales;
+    size_t n;
+    void *out_codes1;        /* mxq_codes_bytes(n, dst_fmt1) bytes */
+    uint8_t *out_scales1;
+    void *out_codes2;        /* mxq_codes_bytes(n, dst_fmt2) bytes */
+    uint8_t *out_scales2;
+} mxq_ss_pair_item;
+
+int mxq_slice_scale_pair_batched(const mxq_ss_pair_item *items, int count, int block, int src_fmt,
+                                 int dst_fmt1, int dst_fmt2, mxq_stream stream);
+
+/*
  * mxq_slice_scale_batched with every tensor's scale bytes written in the tiled order of
  * mxq_tile_scales (the whole-model conversion of Sec. 3.5 handed straight to block-scaled matrix
  * multiplies): item i is a row-major [rows, cols] matrix, and its results are those of
@@ -299,7 +322,7 @@ int mxq_slice_scale_batched(const mxq_ss_item *items, int count, int block,
  * the kernel's parameter space, 256 per launch (more items: more launches); nothing is allocated.
  * Tiled buffers of matrices that do not cover whole tiles are cleared on `stream` first.
  */
-typedef struct {
+typedef struct mxq_ss_tiled_item {
     const void *codes;            /* [in]  device, anchor codes of rows * cols elements */
     const uint8_t *scales;        /* [in]  device, rows * cols / 32 plain scale bytes */
     size_t rows, cols;            /* cols a multiple of 32; rows * cols / 32 below 2^32 */

@@ -47,6 +47,12 @@ class _Item(ctypes.Structure):
                 ("out_codes", ctypes.c_void_p), ("out_scales", ctypes.c_void_p)]
 
 
+class _PairItem(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("n", ctypes.c_size_t),
+                ("out_codes1", ctypes.c_void_p), ("out_scales1", ctypes.c_void_p),
+                ("out_codes2", ctypes.c_void_p), ("out_scales2", ctypes.c_void_p)]
+
+
 class _TiledItem(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("rows", ctypes.c_size_t),
                 ("cols", ctypes.c_size_t), ("out_codes", ctypes.c_void_p), ("out_tiled_scales", ctypes.c_void_p)]
@@ -103,6 +109,8 @@ def load_library() -> ctypes.CDLL:
     L.mxq_slice_scale_tiled_batched.restype = i
     L.mxq_fake_quant_bwd.argtypes = [vp, i, sz, vp, vp]
     L.mxq_slice_scale_batched.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
+    L.mxq_slice_scale_pair_batched.argtypes = [ctypes.POINTER(_PairItem), i, i, i, i, i, vp]
+    L.mxq_slice_scale_pair_batched.restype = i
     L.mxq_slice_scale_batched_static.argtypes = [ctypes.POINTER(_Item), i, i, i, i, vp]
     L.mxq_slice_scale_batched_static.restype = i
     for name in ("mxq_quantize", "mxq_slice_scale", "mxq_dequantize", "mxq_fake_quant", "mxq_fake_quant_bwd",
@@ -487,6 +495,34 @@ def slice_scale_batched(items, src_fmt: str, dst_fmt: str, block: int = 32, stre
     table = items if isinstance(items, ItemTable) else ItemTable(items)
     _check(L.mxq_slice_scale_batched(table.array, len(table), block, FORMATS[src_fmt], FORMATS[dst_fmt],
                                      _stream(stream)), "mxq_slice_scale_batched")
+
+
+class PairItemTable:
+    """A marshalled mxq_ss_pair_item array over (codes, scales, n, out_codes1, out_scales1, out_codes2,
+    out_scales2) tuples that persist (keeps the tensors alive)."""
+
+    def __init__(self, items):
+        self.tensors = list(items)
+        self.array = (_PairItem * len(self.tensors))()
+        for k, (c, s, n, c1, s1, c2, s2) in enumerate(self.tensors):
+            self.array[k] = _PairItem(_dev(c, "codes"), _dev(s, "scales"), n, _dev(c1, "out_codes1"), _dev(s1, "out_scales1"),
+                                      _dev(c2, "out_codes2"), _dev(s2, "out_scales2"))
+
+    def __len__(self):
+        return len(self.tensors)
+
+
+def make_pair_items(items) -> PairItemTable:
+    """Marshal (codes, scales, n, out_codes1, out_scales1, out_codes2, out_scales2) tuples into an mxq_ss_pair_item array."""
+    return PairItemTable(items)
+
+
+def slice_scale_pair_batched(items, src_fmt: str, dst_fmt1: str, dst_fmt2: str, block: int = 32, stream=None) -> None:
+    """mxq_slice_scale_pair_batched: every anchor of a set of tensors to two lower formats, one read of the anchor."""
+    L = load_library()
+    table = items if isinstance(items, PairItemTable) else PairItemTable(items)
+    _check(L.mxq_slice_scale_pair_batched(table.array, len(table), block, FORMATS[src_fmt], FORMATS[dst_fmt1],
+                                          FORMATS[dst_fmt2], _stream(stream)), "mxq_slice_scale_pair_batched")
 
 
 class TiledItemTable:

@@ -422,5 +422,82 @@ int mxq_slice_scale_batched(const mxq_ss_item* items, int count, int block, int 
     return MXQ_OK;
 }
 
+int mxq_slice_scale_pair_batched(const mxq_ss_pair_item* items, int count, int block, int src_fmt, int dst_fmt1,
+                                 int dst_fmt2, mxq_stream stream)
+{
+    if (!valid_format(src_fmt) || !valid_format(dst_fmt1) || !valid_format(dst_fmt2)) return MXQ_ERR_FORMAT;
+    if (!valid_block(block)) return MXQ_ERR_BLOCK;
+    if (block < 32) return MXQ_ERR_BLOCK;
+    if (!ss_pair_ok(src_fmt, dst_fmt1) || !ss_pair_ok(src_fmt, dst_fmt2)) return MXQ_ERR_PAIR;
+    if (count < 0) return MXQ_ERR_SIZE;
+    if (count == 0) return MXQ_OK;
+    if (!items) return MXQ_ERR_NULL;
+    for (int i = 0; i < count; ++i) {
+        const mxq_ss_pair_item& it = items[i];
+        if (it.n % (size_t)block || it.n % 32) return MXQ_ERR_SIZE;
+        if (it.n == 0) continue;
+        if (!it.codes || !it.scales || !it.out_codes1 || !it.out_scales1 || !it.out_codes2 || !it.out_scales2)
+            return MXQ_ERR_NULL;
+        if (!aligned(it.codes, 32) || !aligned(it.out_codes1, 32) || !aligned(it.out_codes2, 32) ||
+            !aligned(it.scales, 16) || !aligned(it.out_scales1, 16) || !aligned(it.out_scales2, 16))
+            return MXQ_ERR_ALIGN;
+    }
+    if (!slice_scale2_is_fused(src_fmt, dst_fmt1, dst_fmt2)) {
+        // no fused kernel for this pair of targets: one single-target batched pass each
+        std::vector<mxq_ss_item> one((size_t)count);
+        for (int t = 0; t < 2; ++t) {
+            for (int i = 0; i < count; ++i) {
+                mxq_ss_item& o = one[(size_t)i];
+                o.codes = items[i].codes;
+                o.scales = items[i].scales;
+                o.n = items[i].n;
+                o.out_codes = t ? items[i].out_codes2 : items[i].out_codes1;
+                o.out_scales = t ? items[i].out_scales2 : items[i].out_scales1;
+            }
+            if (int rc = mxq_slice_scale_batched(one.data(), count, block, src_fmt, t ? dst_fmt2 : dst_fmt1, stream)) return rc;
+        }
+        return MXQ_OK;
+    }
+    MXQ_DEBUG_SCOPE();
+    for (int i = 0; i < count; ++i) {
+        MXQ_DEBUG_EXPECT(items[i].codes, items[i].n * (size_t)fmt_info(src_fmt).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].scales, items[i].n / (size_t)block);
+        MXQ_DEBUG_EXPECT(items[i].out_codes1, items[i].n * (size_t)fmt_info(dst_fmt1).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].out_scales1, items[i].n / (size_t)block);
+        MXQ_DEBUG_EXPECT(items[i].out_codes2, items[i].n * (size_t)fmt_info(dst_fmt2).bits / 8);
+        MXQ_DEBUG_EXPECT(items[i].out_scales2, items[i].n / (size_t)block);
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<Ss2DeviceItem> chunk;
+    chunk.reserve(kSs2BatchItemsMax);
+    size_t tiles = 0;
+    auto flush = [&]() -> int {
+        if (chunk.empty()) return MXQ_OK;
+        const int rc = launch_slice_scale2_batched(chunk.data(), (int)chunk.size(), tiles, src_fmt, dst_fmt1, dst_fmt2, s);
+        chunk.clear();
+        tiles = 0;
+        return rc;
+    };
+    for (int i = 0; i < count; ++i) {
+        const mxq_ss_pair_item& it = items[i];
+        if (it.n == 0) continue;
+        Ss2DeviceItem d;
+        d.codes = static_cast<const uint8_t*>(it.codes);
+        d.scales = it.scales;
+        d.out_codes1 = static_cast<uint8_t*>(it.out_codes1);
+        d.out_scales1 = it.out_scales1;
+        d.out_codes2 = static_cast<uint8_t*>(it.out_codes2);
+        d.out_scales2 = it.out_scales2;
+        d.nunits = it.n / 32;
+        d.nscales = it.n / (size_t)block;
+        d.tile_begin = tiles;
+        tiles += ss2_batched_tiles(d.nunits);
+        chunk.push_back(d);
+        if ((int)chunk.size() == kSs2BatchItemsMax)
+            if (int rc = flush()) return rc;
+    }
+    return flush();
+}
+
 }  // extern "C"
 #pragma GCC visibility pop

@@ -968,31 +968,18 @@ slice_scale_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
 // lower precisions wanted at once).  Per element 1.03 bytes are read once instead of twice.
 // (Left to itself the compiler gives this kernel 64 - 71 registers, 7 CTAs per SM; asked for 12 CTAs it
 // finds 40 without spilling, and the launch is 2 % shorter.)
-template <class FH, class FL1, class FL2, int U, int THREADS>
-__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
-slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits, size_t nscales,
-                    uint8_t* __restrict__ out_codes1, uint8_t* __restrict__ out_scales1,
-                    uint8_t* __restrict__ out_codes2, uint8_t* __restrict__ out_scales2)
+// One warp tile of the two-target conversion; shared by the single-tensor and the batched kernels.
+template <class FH, class FL1, class FL2, int U>
+__device__ __forceinline__ void slice_scale2_tile(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                                  size_t nunits, size_t nscales, uint8_t* __restrict__ out_codes1,
+                                                  uint8_t* __restrict__ out_scales1, uint8_t* __restrict__ out_codes2,
+                                                  uint8_t* __restrict__ out_scales2, size_t tile, uint8_t* stage1,
+                                                  uint8_t* stage2)
 {
-    pdl_release();
     constexpr int IB = 4 * FH::bits, NWI = IB / 4;
     constexpr int OB1 = 4 * FL1::bits, OB2 = 4 * FL2::bits;
     constexpr int de1 = FH::emax - FL1::emax, de2 = FH::emax - FL2::emax;
-    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     const size_t u0 = tile * (32 * U) + (threadIdx.x & 31);
-    uint8_t* stage1 = nullptr;
-    uint8_t* stage2 = nullptr;
-    if constexpr (StagedTile<OB1>::use) {
-        __shared__ __align__(128) uint8_t area1[(THREADS / 32) * 32 * U * OB1];
-        stage1 = area1 + (threadIdx.x >> 5) * (32 * U * OB1);
-    }
-    if constexpr (StagedTile<OB2>::use) {
-        __shared__ __align__(128) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
-        stage2 = area2 + (threadIdx.x >> 5) * (32 * U * OB2);
-    }
-    prefetch_tile<U, IB>(codes, tile, nunits);
-    pdl_acquire();
-    if (tile * (32 * U) >= nunits) return;                     // whole warps leave together
     uint32_t w[U][NWI];
     uint32_t sb[U];
 #pragma unroll
@@ -1051,6 +1038,41 @@ slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict
     }
 }
 
+// The two staging areas of the calling warp (null where the target's pieces are stored directly).
+// Must be called by every thread of the CTA, outside divergent code.
+template <class FL1, class FL2, int U, int THREADS>
+__device__ __forceinline__ void slice_scale2_stages(uint8_t*& stage1, uint8_t*& stage2)
+{
+    constexpr int OB1 = 4 * FL1::bits, OB2 = 4 * FL2::bits;
+    stage1 = nullptr;
+    stage2 = nullptr;
+    if constexpr (StagedTile<OB1>::use) {
+        __shared__ __align__(128) uint8_t area1[(THREADS / 32) * 32 * U * OB1];
+        stage1 = area1 + (threadIdx.x >> 5) * (32 * U * OB1);
+    }
+    if constexpr (StagedTile<OB2>::use) {
+        __shared__ __align__(128) uint8_t area2[(THREADS / 32) * 32 * U * OB2];
+        stage2 = area2 + (threadIdx.x >> 5) * (32 * U * OB2);
+    }
+}
+
+template <class FH, class FL1, class FL2, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
+slice_scale2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales, size_t nunits, size_t nscales,
+                    uint8_t* __restrict__ out_codes1, uint8_t* __restrict__ out_scales1,
+                    uint8_t* __restrict__ out_codes2, uint8_t* __restrict__ out_scales2)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t *stage1, *stage2;
+    slice_scale2_stages<FL1, FL2, U, THREADS>(stage1, stage2);
+    prefetch_tile<U, 4 * FH::bits>(codes, tile, nunits);
+    pdl_acquire();
+    if (tile * (32 * U) >= nunits) return;                     // whole warps leave together
+    slice_scale2_tile<FH, FL1, FL2, U>(codes, scales, nunits, nscales, out_codes1, out_scales1, out_codes2, out_scales2,
+                                       tile, stage1, stage2);
+}
+
 // Device-side item of the batched conversion (one tensor), with its place in the flattened
 // tile space of the whole batch.
 struct SsDeviceItem {
@@ -1106,6 +1128,45 @@ slice_scale_batched_param_kernel(const __grid_constant__ SsItemBlock<K> blk, int
     if (tile >= total_tiles) return;
     slice_scale_tile<FH, FL, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes, t.out_scales, tile - t.tile_begin,
                                 stage);
+}
+
+// Two targets from one read of every anchor of a set of tensors (the whole-model conversion of Sec. 3.5
+// for a deployment that serves two lower precisions at once): items of 72 bytes, 256 per launch.
+struct Ss2DeviceItem {
+    const uint8_t* codes;
+    const uint8_t* scales;
+    uint8_t* out_codes1;
+    uint8_t* out_scales1;
+    uint8_t* out_codes2;
+    uint8_t* out_scales2;
+    size_t nunits;
+    size_t nscales;
+    size_t tile_begin;
+};
+
+template <int K>
+struct Ss2ItemBlock {
+    Ss2DeviceItem items[K];
+    TileIndex index;
+};
+
+// (The item's six pointers live in registers here.  Measured over the 224-tensor weight set with 6 / 8 / 10 / 12
+// resident CTAs: 10 -- 48 registers, 12 - 20 bytes of spills in the MXFP variants -- is the fastest for the
+// MXFP pair (2.42 ms against 2.60 at 8 and 3.13 at 12) and within 2 % of the best for the MXINT pair.)
+template <class FH, class FL1, class FL2, int U, int THREADS, int K>
+__global__ void __launch_bounds__(THREADS, 10)
+slice_scale2_batched_kernel(const __grid_constant__ Ss2ItemBlock<K> blk, int count, size_t total_tiles)
+{
+    pdl_release();
+    const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
+    uint8_t *stage1, *stage2;
+    slice_scale2_stages<FL1, FL2, U, THREADS>(stage1, stage2);
+    const Ss2DeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
+    if (tile < total_tiles) prefetch_tile<U, 4 * FH::bits>(t.codes, tile - t.tile_begin, t.nunits);
+    pdl_acquire();
+    if (tile >= total_tiles) return;
+    slice_scale2_tile<FH, FL1, FL2, U>(t.codes, t.scales, t.nunits, t.nscales, t.out_codes1, t.out_scales1, t.out_codes2,
+                                       t.out_scales2, tile - t.tile_begin, stage1, stage2);
 }
 
 // The batched conversion with every tensor's scale bytes written in the tiled order (block 32): the

@@ -31,6 +31,14 @@ int launch_slice_scale(const void* codes, const uint8_t* scales, size_t n, int b
 int launch_slice_scale2(const void* codes, const uint8_t* scales, size_t n, int block, int src_fmt, int dst_fmt1,
                         int dst_fmt2, void* out_codes1, uint8_t* out_scales1, void* out_codes2, uint8_t* out_scales2,
                         cudaStream_t stream);
+// The two-target conversion over up to kSs2BatchItemsMax tensors in one launch (items: a HOST array with
+// tile_begin filled in); MXQ_ERR_PAIR when the pair of targets has no fused instantiation.
+struct Ss2DeviceItem;
+constexpr int kSs2BatchItemsMax = 256;
+int launch_slice_scale2_batched(const Ss2DeviceItem* items_host, int count, size_t total_tiles, int src_fmt, int dst_fmt1,
+                                int dst_fmt2, cudaStream_t stream);
+bool slice_scale2_is_fused(int src_fmt, int dst_fmt1, int dst_fmt2);
+size_t ss2_batched_tiles(size_t nunits);
 // The same two operations with the scale bytes written in 128 x 4 tiles (block 32, kblocks block-columns
 // per row); the caller has zeroed the tiled buffer when the matrix leaves part of a tile uncovered.
 int launch_quantize_tiled(const void* src, int dtype, size_t n, int fmt, void* codes, uint8_t* tiled,

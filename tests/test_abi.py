@@ -148,6 +148,17 @@ def test_argument_checks_answer_on_the_host(L):
     assert dqb((_DqItem * 1)(_DqItem(A, A, 16, A)), 1, F["int4"], 16, 1, None) == E_SIZE      # packed codes: multiples of 32
     assert dqb((_DqItem * 1)(_DqItem(A, None, 64, A)), 1, F["int4"], 32, 1, None) == E_NULL
     assert dqb((_DqItem * 1)(_DqItem(A, A + 8, 64, A)), 1, F["int4"], 32, 1, None) == E_ALIGN
+    from paper_2604_00529_b200.binding import _PairItem
+    pb = L.mxq_slice_scale_pair_batched             # (items, count, block, src, dst1, dst2, stream)
+    assert pb(None, 0, 32, F["int8"], F["int6"], F["int4"], None) == OK
+    assert pb(None, 2, 32, F["int8"], F["int6"], F["int4"], None) == E_NULL
+    assert pb(None, -1, 32, F["int8"], F["int6"], F["int4"], None) == E_SIZE
+    assert pb(None, 2, 16, F["int8"], F["int6"], F["int4"], None) == E_BLOCK
+    assert pb(None, 2, 32, F["int8"], F["int6"], F["e2m1"], None) == E_PAIR
+    assert pb(None, 2, 32, F["int8"], 44, F["int4"], None) == E_FORMAT
+    assert pb((_PairItem * 1)(_PairItem(A, A, 65, A, A, A, A)), 1, 32, F["int8"], F["int6"], F["int4"], None) == E_SIZE
+    assert pb((_PairItem * 1)(_PairItem(A, A, 64, A, A, None, A)), 1, 32, F["int8"], F["int6"], F["int4"], None) == E_NULL
+    assert pb((_PairItem * 1)(_PairItem(A, A, 64, A, A, A, A + 8)), 1, 32, F["int8"], F["int6"], F["int4"], None) == E_ALIGN
     bw = L.mxq_fake_quant_bwd
     assert bw(A, 1, 64, A, None) == OK                                       # in place: no launch
     assert bw(A, 1, 64, None, None) == E_NULL

@@ -370,6 +370,38 @@ def test_fake_quant_batched_matches_oracle(count, bf16):
         assert bits_equal(got, want), first_diff(got, want)
 
 
+@pytest.mark.parametrize("count", [1, 5, 256, 257, 600])
+@pytest.mark.parametrize("src,dst1,dst2,block", [("int8", "int6", "int4", 32), ("e4m3", "e2m1", "e2m3", 32),
+                                                  ("e4m3", "e3m2", "e2m1", 64), ("e4m3", "e2m3", "e3m2", 128),
+                                                  ("int8", "int7", "int3", 32), ("e4m3", "e3m3", "e2m2", 32)])
+def test_slice_scale_pair_batched_matches_oracle(count, src, dst1, dst2, block):
+    """Two targets from one read of every anchor of a set of tensors: fused pairs (both orders of the
+    targets) and pairs that fall back to two passes; counts on both sides of the 256-tensor launch limit;
+    all byte values as codes and as scale bytes."""
+    rng = np.random.default_rng(count * 7 + block)
+    nblks = rng.integers(1, 30, count) * (block // 32)
+    if count <= 5:
+        nblks[0] = 2051 * (block // 32)
+    ins, outs = [], []
+    for nb in nblks:
+        n = int(nb) * 32
+        codes = rng.integers(0, 256, n).astype(np.uint8)
+        scales = rng.integers(0, 256, n // block).astype(np.uint8)
+        o = [Guarded(mxq.codes_bytes(n, dst1)), Guarded(n // block), Guarded(mxq.codes_bytes(n, dst2)), Guarded(n // block)]
+        ins.append((codes, scales, n))
+        outs.append(o)
+    items = [(to_dev(c), to_dev(s), n, o[0].view, o[1].view, o[2].view, o[3].view) for (c, s, n), o in zip(ins, outs)]
+    mxq.slice_scale_pair_batched(items, src, dst1, dst2, block)
+    torch.cuda.synchronize()
+    for k, ((c, s, n), o) in enumerate(zip(ins, outs)):
+        for g in o:
+            g.check()
+        for dst, oc, os_ in ((dst1, o[0], o[1]), (dst2, o[2], o[3])):
+            wc, ws = orc.slice_scale(c, s, src, dst, block)
+            assert bits_equal(to_host(os_.view), ws), (k, dst)
+            assert bits_equal(to_host(oc.view), orc.pack(wc, orc.bits(dst))), (k, dst, first_diff(to_host(oc.view), orc.pack(wc, orc.bits(dst))))
+
+
 @pytest.mark.parametrize("count", [1, 6, 512, 513, 1030])
 @pytest.mark.parametrize("fmt,bf16,block", [("int8", True, 32), ("e4m3", False, 32), ("int6", True, 64), ("e2m1", False, 16),
                                              ("int7", True, 32), ("e3m3", True, 128)])
