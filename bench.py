@@ -955,7 +955,8 @@ def run_cuda(args):
         "gpu_launches": headline_launches,
         "gpu_launches_all_workloads": headline_launches + bench.launches,
         "roofline": {"bound": "hbm", "kernel": top_name, "achieved": round(top_gbs, 1), "peak": peak, "unit": "GB/s",
-                     "frac": round(top_gbs / peak, 4), "peak_kind": peak_kind, "traffic": traffic,
+                     "frac": round(top_gbs / peak, 4), "faster_than_the_copy_peak": bool(top_gbs > peak),
+                     "peak_kind": peak_kind, "traffic": traffic,
                      "bytes_per_launch": int(top_bpe * total_elems), "ms_per_launch": round(top_ms, 4),
                      "ncu_dram_pct_of_peak": dram_pct,
                      "note": "achieved counts algorithmic bytes over the CUDA-event duration inside the timed steps; "

@@ -597,13 +597,15 @@ def test_two_streams_run_independent_conversions():
 
 
 @pytest.mark.parametrize("nblk", [4096, 1 << 16, 1 << 19])
-def test_dependent_chain_reusing_buffers_reads_fresh_data(nblk):
+@pytest.mark.parametrize("anchor,low", [("e4m3", "e2m1"), ("e4m3", "e2m3"), ("int8", "int6"), ("int8", "int7")])
+def test_dependent_chain_reusing_buffers_reads_fresh_data(nblk, anchor, low):
     """quantize -> slice_scale -> dequantize -> fake-quant in place, eight rounds back to back on ONE
     stream, every round with new input but the SAME intermediate buffers and no host synchronisation in
     between.  Each kernel starts while its producer is still running (programmatic dependent launch) and
     prefetches its input lines before it waits for the producer; what it then reads must be what the
     producer wrote in this round, not the previous round's bytes.  Sizes: less than one wave of CTAs, a
-    few waves, many waves."""
+    few waves, many waves.  The 6- and 7-bit targets leave their kernel as bulk copies out of shared memory: the
+    consumer must see those bytes too."""
     n = nblk * 32
     rounds = 8
     base = inputs.to_bf16_bits(_mixed_f32(nblk + rounds, 77))
@@ -611,24 +613,25 @@ def test_dependent_chain_reusing_buffers_reads_fresh_data(nblk):
     xs = [to_dev(x) for x in xs_host]
     codes = torch.empty(n, dtype=torch.uint8, device="cuda")
     scales = torch.empty(nblk, dtype=torch.uint8, device="cuda")
-    low_c = torch.empty(n // 2, dtype=torch.uint8, device="cuda")
+    bl = orc.bits(low)
+    low_c = torch.empty(n * bl // 8, dtype=torch.uint8, device="cuda")
     low_s = torch.empty(nblk, dtype=torch.uint8, device="cuda")
     v = torch.empty(n, dtype=torch.bfloat16, device="cuda")
     kept = []
     torch.cuda.synchronize()
     for r in range(rounds):
-        mxq.quantize(xs[r], "e4m3", 32, codes, scales)
-        mxq.slice_scale(codes, scales, n, "e4m3", "e2m1", 32, low_c, low_s)
-        mxq.dequantize(low_c, low_s, n, "e2m1", 32, dst=v)
+        mxq.quantize(xs[r], anchor, 32, codes, scales)
+        mxq.slice_scale(codes, scales, n, anchor, low, 32, low_c, low_s)
+        mxq.dequantize(low_c, low_s, n, low, 32, dst=v)
         mxq.fake_quant(v, "e2m3", 32, mxq.FQ_DIRECT, dst=v)                # in place, on what was just written
         kept.append((mxq.fake_quant_bwd(low_c.view(torch.bfloat16)), mxq.fake_quant_bwd(v)))   # stream-ordered copies
     torch.cuda.synchronize()
     for r in (0, 3, rounds - 1) if nblk > 4096 else range(rounds):
-        oc, os_ = orc.quantize(xs_host[r], "e4m3")
-        wc, ws = orc.slice_scale(oc, os_, "e4m3", "e2m1")
-        want_v = orc.dequantize(wc, ws, "e2m1", out_dtype=orc.BF16)
+        oc, os_ = orc.quantize(xs_host[r], anchor)
+        wc, ws = orc.slice_scale(oc, os_, anchor, low)
+        want_v = orc.dequantize(wc, ws, low, out_dtype=orc.BF16)
         got_c, got_v = kept[r]
-        assert bits_equal(to_host(got_c.view(torch.uint8)), orc.pack(wc, 4)), (r, "codes")
+        assert bits_equal(to_host(got_c.view(torch.uint8)), orc.pack(wc, bl)), (r, "codes")
         assert bits_equal(to_host(got_v), orc.fake_quant(want_v, "e2m3", mode=orc.FQ_DIRECT)), (r, "values")
 
 
