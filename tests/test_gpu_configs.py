@@ -147,6 +147,73 @@ def test_workload3_whole_model_batched_conversion(anchor, targets):
         del outs, table
 
 
+def test_workload3_headline_step_in_the_launch_configuration_of_the_bench():
+    """The ten launches of the bench's headline step, each over all 224 tensors of the weight set laid
+    out in one arena per stream as the bench lays them out: quantize_batched to both anchors,
+    slice_scale_batched to the 4-bit targets, dequantize_batched, fake_quant_batched (E2M3 through the
+    anchor) and the straight-through copy of the whole arena.  Four layers are drawn on the host, the
+    others are device copies of them in turn; every tensor is checked on sampled block runs (first and
+    last blocks among them) against the oracle run on the host bits of the same elements."""
+    drawn = (0, 13, 31, 7)
+    shapes = inputs.llama8b_shapes()
+    sizes = [r * c for *_, r, c in shapes]
+    total = sum(sizes)
+    layer_elems = sum(r * c for _, r, c in inputs.LLAMA8B_LAYER)
+    host = [np.concatenate([inputs.llama8b_tensor(layer, idx) for idx in range(len(inputs.LLAMA8B_LAYER))]) for layer in drawn]
+    w = torch.empty(total, dtype=torch.bfloat16, device="cuda")
+    for li, bits in enumerate(host):
+        w[li * layer_elems:(li + 1) * layer_elems].copy_(to_dev(bits))
+    for l in range(len(drawn), inputs.LLAMA8B_LAYERS):
+        src = (l % len(drawn)) * layer_elems
+        w[l * layer_elems:(l + 1) * layer_elems].copy_(w[src:src + layer_elems])
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+
+    def host_bits(k, lo, hi):                       # elements [lo, hi) of tensor k
+        layer = shapes[k][0]
+        base = int(offs[k]) - layer * layer_elems
+        return host[layer % len(drawn)][base + lo:base + hi]
+
+    u8 = dict(dtype=torch.uint8, device="cuda")
+    T = range(len(sizes))
+    sl = lambda buf, k, bits=8: buf[int(offs[k]) * bits // 8:int(offs[k + 1]) * bits // 8]
+    ss = lambda buf, k: buf[int(offs[k]) // BLOCK:int(offs[k + 1]) // BLOCK]
+    deq = torch.empty(total, dtype=torch.bfloat16, device="cuda")
+    for anchor, low in (("int8", "int4"), ("e4m3", "e2m1")):
+        ac, as_ = torch.empty(total, **u8), torch.empty(total // BLOCK, **u8)
+        lc, ls = torch.empty(total // 2, **u8), torch.empty(total // BLOCK, **u8)
+        mxq.quantize_batched([(w[int(offs[k]):int(offs[k + 1])], sl(ac, k), ss(as_, k)) for k in T], anchor, BLOCK)
+        mxq.slice_scale_batched([(sl(ac, k), ss(as_, k), sizes[k], sl(lc, k, 4), ss(ls, k)) for k in T], anchor, low, BLOCK)
+        mxq.dequantize_batched([(sl(lc, k, 4), ss(ls, k), sizes[k], deq[int(offs[k]):int(offs[k + 1])]) for k in T], low, BLOCK)
+        torch.cuda.synchronize()
+        for k in T:
+            for lo, hi in sample_runs(sizes[k] // BLOCK, 1, 256, k):
+                x = host_bits(k, lo * BLOCK, hi * BLOCK)
+                wc, ws = orc.quantize(x, anchor, BLOCK)
+                assert bits_equal(dev_slice(ss(as_, k), lo, hi), ws), (anchor, k, lo)
+                assert bits_equal(dev_slice(sl(ac, k), lo * BLOCK, hi * BLOCK), orc.pack(wc, 8)), (anchor, k, lo)
+                w4, s4 = orc.slice_scale(wc, ws, anchor, low, BLOCK)
+                assert bits_equal(dev_slice(sl(lc, k, 4), lo * BLOCK // 2, hi * BLOCK // 2), orc.pack(w4, 4)), (low, k, lo)
+                assert bits_equal(dev_slice(ss(ls, k), lo, hi), s4), (low, k, lo)
+                want = orc.dequantize(w4, s4, low, BLOCK, orc.BF16)
+                got = dev_slice(deq[int(offs[k]):int(offs[k + 1])], lo * BLOCK, hi * BLOCK)
+                assert bits_equal(got, want), (low, k, lo, first_diff(got, want))
+        del ac, as_, lc, ls
+    fq = deq                                        # reuse the arena
+    mxq.fake_quant_batched([(w[int(offs[k]):int(offs[k + 1])], fq[int(offs[k]):int(offs[k + 1])]) for k in T], "e2m3", BLOCK,
+                           mxq.FQ_VIA_ANCHOR)
+    torch.cuda.synchronize()
+    for k in T:
+        for lo, hi in sample_runs(sizes[k] // BLOCK, 1, 256, 1000 + k):
+            want = orc.fake_quant(host_bits(k, lo * BLOCK, hi * BLOCK), "e2m3", BLOCK, orc.FQ_VIA_ANCHOR)
+            got = dev_slice(fq[int(offs[k]):int(offs[k + 1])], lo * BLOCK, hi * BLOCK)
+            assert bits_equal(got, want), ("fake_quant", k, lo, first_diff(got, want))
+    grad = torch.empty_like(fq)
+    mxq.fake_quant_bwd(fq, grad)                    # 6.98 G elements in one call
+    torch.cuda.synchronize()
+    for lo in (0, total // 3, total - (1 << 20)):
+        assert torch.equal(grad[lo:lo + (1 << 20)].view(torch.int16), fq[lo:lo + (1 << 20)].view(torch.int16))
+
+
 # ---------------------------------------------------------------------------------------------
 # workload 4: BF16 activations [8 x 4096, 4096] with hot channels; per call a format sampled by seed,
 # both routes (direct, through the anchor), and the straight-through backward
