@@ -66,6 +66,14 @@ __device__ __forceinline__ void st256(void* p, const uint32_t (&w)[8])
                  : "memory");
 }
 
+// 32 bytes of one repeated word (the quiet-NaN fill of a poisoned block): a store of its own, under the
+// block's predicate, instead of eight selects in front of the ordinary store.
+__device__ __forceinline__ void st256_splat(void* p, uint32_t v)
+{
+    MXQ_CHECKED(p, 32, return)
+    asm volatile("st.global.v8.u32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" :: "l"(p), "r"(v) : "memory");
+}
+
 // ---- single bytes (the scale streams) -------------------------------------------------------
 
 __device__ __forceinline__ uint32_t ld_u8(const uint8_t* p)

@@ -534,11 +534,10 @@ __device__ __forceinline__ void fake_quant_tile(const uint8_t* src, size_t nunit
                 out[I] = pack_bf16x2(y0, y1);
             }
         });
-        if (s.byte == 0xFFu) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) out[j] = T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u;
+        if (unit < nunits) {
+            if (s.byte == 0xFFu) st256_splat(dst + unit * 32, T::size == 4 ? 0x7FC00000u : 0x7FC07FC0u);   // poisoned block
+            else st256(dst + unit * 32, out);
         }
-        if (unit < nunits) st256(dst + unit * 32, out);
     }
 }
 
