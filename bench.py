@@ -154,7 +154,17 @@ class ClockSampler:
     REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"),
                (0x4, "sw_power_cap"))
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, uuid: str = None):
+        # `index` counts the devices this process sees; NVML counts all of the machine's, so the device
+        # is looked up by UUID where torch gives one, else through CUDA_VISIBLE_DEVICES
+        self.uuid = uuid
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        ids = [v.strip() for v in vis.split(",") if v.strip()]
+        if uuid is None and index < len(ids):
+            if ids[index].isdigit():
+                index = int(ids[index])
+            elif ids[index].startswith("GPU-"):
+                self.uuid = ids[index]
         self.index = index
         self.samples = []                   # (t, sm_mhz, reasons bitmask)
         self.max_mhz = None
@@ -166,7 +176,13 @@ class ClockSampler:
         try:
             import pynvml
             pynvml.nvmlInit()
-            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            if self.uuid:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(self.uuid.encode())
+                except TypeError:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(self.uuid)
+            else:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
             self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
             reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 getattr(pynvml, "nvmlDeviceGetCurrentClocksThrottleReasons")
@@ -185,7 +201,7 @@ class ClockSampler:
             q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                  "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
             try:
-                proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
+                proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid or str(self.index), "--query-gpu=" + q,
                                          "--format=csv,noheader,nounits", "-lms", "100"],
                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             except OSError:
@@ -836,7 +852,8 @@ def run_cuda(args):
     import paper_2604_00529_b200 as mxq
     mxq.load_library()
     peak, peak_kind = peaks()
-    sampler = ClockSampler(local)
+    uuid = getattr(torch.cuda.get_device_properties(local), "uuid", None)
+    sampler = ClockSampler(local, "GPU-%s" % uuid if uuid is not None else None)
     sampler.start()
     bench = Bench(torch, sampler, peak, peak_kind)
     t_begin = time.perf_counter()
