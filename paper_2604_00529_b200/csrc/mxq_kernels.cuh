@@ -609,7 +609,7 @@ struct FqItemBlock {
     TileIndex index;
 };
 
-template <class T, class F, int BLOCK, int MODE, int U, int THREADS, int K>
+template <class T, class F, int BLOCK, int MODE, int U, int R, int THREADS, int K>
 __global__ void __launch_bounds__(THREADS, 14)
 fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count, size_t total_tiles)
 {
@@ -617,10 +617,18 @@ fake_quant_batched_kernel(const __grid_constant__ FqItemBlock<K> blk, int count,
     const size_t tile = (size_t)blockIdx.x * (THREADS / 32) + (threadIdx.x >> 5);
     // the item table is a kernel parameter, so the lookup may run before the dependency wait
     const FqDeviceItem& t = blk.items[tile < total_tiles ? find_item(blk.items, blk.index, tile) : 0];
-    if (tile < total_tiles) prefetch_tile<U, 32>(t.src, tile - t.tile_begin, t.nunits);
+    // A tile of the batch is R consecutive warp tiles of ONE tensor, converted one after the other: the
+    // lookup above (some 25 instructions per thread) is paid once per R * 32 * U lane units.
+    const size_t first = (tile - t.tile_begin) * R;
+    if (tile < total_tiles) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) prefetch_tile<U, 32>(t.src, first + r, t.nunits);
+    }
     pdl_acquire();
     if (tile >= total_tiles) return;                      // whole warps leave together
-    fake_quant_tile<T, F, BLOCK, MODE, U>(t.src, t.nunits, t.dst, tile - t.tile_begin);
+#pragma unroll 1
+    for (int r = 0; r < R; ++r)
+        if ((first + r) * (32 * U) < t.nunits) fake_quant_tile<T, F, BLOCK, MODE, U>(t.src, t.nunits, t.dst, first + r);
 }
 
 // Q_f (Eq. 1-3) over a whole set of tensors in one launch (the anchor checkpoint of a model, Sec. 3.5:
